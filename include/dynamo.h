@@ -1,0 +1,182 @@
+/*
+ * dynamo.h - C-ABI of the B200-native DynaMo quantized-MoE hot path.
+ *
+ * One MoE layer = one context.  The layer's routed-expert SwiGLU FFN runs over
+ * expert-level mixed-precision weights (each expert bit-packed at its own base
+ * bit-width, group-wise fp16 scale / fp16 zero) combined with the channel-level
+ * dynamic switch: a runtime-selected set of significant input channels per expert
+ * is served at 8-bit precision from the channel cache while the rest stay at the
+ * expert's base precision.
+ *
+ * Conventions
+ *  - Every function returns a dynamo_status (0 = OK).  No exceptions, no global state.
+ *  - "dev" pointers are CUDA device pointers, "host" pointers are ordinary host memory.
+ *  - All device buffers are CALLER-OWNED.  The context owns only host metadata and
+ *    pointers into the caller's arenas; the library never calls cudaMalloc.
+ *  - Calls that touch the device take a cudaStream_t (passed as void*; NULL = the
+ *    legacy default stream), are asynchronous and stream-ordered unless stated.
+ *  - Argument errors are detected on the host BEFORE any launch and leave all state
+ *    unchanged.  Device-side waits are bounded; an expired wait sets a status word
+ *    that dynamo_poll_status reads.
+ *  - One context per layer, externally synchronised (not thread-safe).
+ *  - Shapes: d_model % 256 == 0, d_ff % 128 == 0, group_size in {64, 128},
+ *    1 <= top_k <= 8, n_experts <= 256, n_experts + n_shared <= 264, top_k <= n_experts,
+ *    max_sig <= cache_size <= d_model, max_sig <= 256.
+ *  - MMA operand format is fp16 (codes and activations are exact in it; the hidden
+ *    activation h is rounded to fp16); accumulation is fp32.
+ */
+#ifndef DYNAMO_H_
+#define DYNAMO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DYNAMO_OK = 0,
+    DYNAMO_ERR_NULL = 1,            /* a required pointer is NULL */
+    DYNAMO_ERR_SHAPE = 2,           /* a dimension violates the shape rules above */
+    DYNAMO_ERR_BITS = 3,            /* a bit-width is not one of 2, 3, 4, 8 (shared experts: 8) */
+    DYNAMO_ERR_ALIGN = 4,           /* a device buffer is not 256-byte aligned */
+    DYNAMO_ERR_ARENA_TOO_SMALL = 5, /* weights arena or workspace smaller than dynamo_arena_bytes says */
+    DYNAMO_ERR_INDEX_RANGE = 6,     /* a channel index is outside [0, d_model) or a count outside [0, S] */
+    DYNAMO_ERR_INDEX_DUP = 7,       /* a channel index appears twice / cache_idx not strictly increasing */
+    DYNAMO_ERR_NOT_CACHED = 8,      /* a significant channel is not in that expert's channel cache */
+    DYNAMO_ERR_STATE = 9,           /* call made before dynamo_pack_experts */
+    DYNAMO_ERR_TOKENS = 10,         /* T < 0 or T > max_tokens */
+    DYNAMO_ERR_CUDA = 11,           /* a CUDA runtime call failed */
+    DYNAMO_ERR_TIMEOUT = 12         /* a bounded device-side wait expired (see dynamo_poll_status) */
+} dynamo_status;
+
+typedef struct {
+    int32_t d_model;     /* d: expert input / output width */
+    int32_t d_ff;        /* f: expert hidden width */
+    int32_t n_experts;   /* E: routed experts */
+    int32_t n_shared;    /* E_s: always-on shared experts (8-bit, weight 1), may be 0 */
+    int32_t top_k;       /* k */
+    int32_t group_size;  /* G: quantization group along the input axis, 64 or 128 */
+    int32_t max_sig;     /* S: capacity of one expert's significant-channel set */
+    int32_t cache_size;  /* P: channels per expert kept in the channel cache (candidates) */
+    int32_t max_tokens;  /* largest T a forward may be called with */
+    int32_t renormalize; /* 1: the k routing weights are rescaled to sum to 1 */
+} dynamo_layer_desc;
+
+typedef struct dynamo_ctx dynamo_ctx;
+
+/* Optional device outputs of a forward, for parity checks (any member may be NULL). */
+typedef struct {
+    int32_t* topk_idx;       /* dev int32 [T, k]   chosen experts, descending logit            */
+    float*   topk_w;         /* dev fp32  [T, k]   routing weights                             */
+    int32_t* expert_offsets; /* dev int32 [E + 1]  exclusive scan of per-expert pair counts    */
+    int32_t* perm;           /* dev int32 [T * k]  sorted row -> t*k + j                       */
+} dynamo_debug_out;
+
+enum { DYNAMO_BF16 = 0, DYNAMO_F32 = 1 };                       /* y_dtype */
+enum { DYNAMO_MAT_GATE = 0, DYNAMO_MAT_UP = 1, DYNAMO_MAT_DOWN = 2 };
+enum { DYNAMO_CODES_BASE = 0,      /* base-precision codes and params of the whole matrix          */
+       DYNAMO_CODES_HI_POOL = 1,   /* 8-bit codes of the cached channels (0 elsewhere), 8-bit params */
+       DYNAMO_CODES_HI_ACTIVE = 2  /* as HI_POOL but only the currently significant channels        */ };
+enum { DYNAMO_SWITCH_SELECT = 0,   /* switch = re-point the active list at codes quantized at pack time */
+       DYNAMO_SWITCH_REQUANT = 1   /* switch also re-derives the entering channels' 8-bit codes from the
+                                      bf16 originals in the channel cache (the paper's replace-then-requantize) */ };
+
+/* Create / destroy a layer context.  Host only; needs no GPU.  [layer shape: Section II-A] */
+dynamo_status dynamo_create(const dynamo_layer_desc* desc, dynamo_ctx** out);
+dynamo_status dynamo_destroy(dynamo_ctx* ctx);
+
+/* Bytes the caller must provide for the packed weights arena (persistent layer state:
+ * packed codes, params, channel cache, 8-bit pool, switch tables) and for the workspace
+ * (scratch of pack and forward; may be shared by several layers whose calls are ordered on
+ * one stream).  bits: host int32 [E + E_s], routed experts in {2,3,4,8}, shared experts 8.
+ * Host only. */
+dynamo_status dynamo_arena_bytes(const dynamo_layer_desc* desc, const int32_t* bits,
+                                 size_t* weights_bytes, size_t* workspace_bytes);
+
+/* Offline step: quantize and bit-pack every expert at its assigned bit-width and build the
+ * channel cache.  [Section IV-A: expert-level uniform mixed-precision quantization;
+ * Section V-B: several low-bit codes packed per 32-bit word; Sections IV-B, V-A: cache of the
+ * original channels with (expert, channel) index headers.]
+ *   w_gate, w_up : dev bf16 [E+E_s, f, d] row-major;  w_down : dev bf16 [E+E_s, d, f].
+ *   bits         : host int32 [E+E_s].
+ *   cache_idx    : host int32 [E, P], each row strictly increasing, in [0, d).
+ * Per (row, group of G input indices): scale = fp16((max-min)/(2^b-1)) (1.0 if that rounds to 0),
+ * zero = fp16(min), code = clamp(rint((w-zero)/scale), 0, 2^b-1), all in IEEE double with ties
+ * to even.  For every routed expert with bits < 8 the 8-bit parameters of W_gate/W_up, the 8-bit
+ * codes of the P cached channels and their bf16 originals are stored as well.  The significant
+ * sets are installed empty.  The arenas must stay valid and unmoved while the context is used.
+ * Inputs may be freed once the stream has passed this call. */
+dynamo_status dynamo_pack_experts(dynamo_ctx* ctx, const void* w_gate, const void* w_up, const void* w_down,
+                                  const int32_t* bits, const int32_t* cache_idx,
+                                  void* weights_arena, size_t weights_bytes,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* Runtime channel switch: install the significant-channel set of every routed expert.
+ * [Section IV-B: channel replacement from the cache and requantization; Section V-A: lookup by
+ * (expert, channel) header.]
+ *   sig_idx : host int32 [E, S] (only the first sig_cnt[e] entries of a row are read)
+ *   sig_cnt : host int32 [E], each in [0, S].
+ * The state afterwards depends only on the sets given (not on history).  Channels must be in the
+ * expert's cache (ERR_NOT_CACHED), in range (ERR_INDEX_RANGE), unique (ERR_INDEX_DUP); on any
+ * error the previous sets stay installed.  Base codes and params are never touched.  For experts
+ * with 8-bit base precision the set is a no-op.  Stream-ordered: a switch enqueued between two
+ * forwards takes effect exactly between them. */
+dynamo_status dynamo_set_channel_switch(dynamo_ctx* ctx, const int32_t* sig_idx, const int32_t* sig_cnt,
+                                        void* stream);
+
+/* A whole switch event (all layers of a stack) in one upload and one launch; all-or-nothing.
+ * sig_idx host int32 [n_layers, E, S], sig_cnt host int32 [n_layers, E]; n_layers <= 64; all
+ * layers must share shape and workspace. */
+dynamo_status dynamo_set_channel_switch_many(dynamo_ctx* const* ctxs, int32_t n_layers,
+                                             const int32_t* sig_idx, const int32_t* sig_cnt, void* stream);
+
+/* Select how a switch brings entering channels to 8-bit (DYNAMO_SWITCH_*; default SELECT).
+ * Both give bit-identical state. */
+dynamo_status dynamo_set_switch_mode(dynamo_ctx* ctx, int32_t mode);
+
+/* Forward of the layer: router top-k -> token permutation -> mixed-precision grouped SwiGLU FFN
+ * with the significant-channel correction -> weighted un-permute.  [Section II-A: Top-K expert
+ * selection, one-to-many dispatch; Section V-B: packed load, dequantize, tensor-core MMA, fused.]
+ *   x             : dev bf16 [T, d]
+ *   router_logits : dev fp32 [T, E]   (the router GEMM is outside this path)
+ *   y             : dev [T, d], bf16 or fp32 per y_dtype
+ * topk = the k largest logits (ties -> lower index), weights = softmax over all E restricted to
+ * the chosen k (rescaled to sum 1 if renormalize).  y[t] = sum_j w[t,j] * FFN_{e_j}(x[t]) +
+ * sum_shared FFN_s(x[t]), summed in fp32 in that order.  T = 0 is a no-op. */
+dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* router_logits, int32_t T,
+                                 void* y, int32_t y_dtype, const dynamo_debug_out* dbg, void* stream);
+
+/* Same forward with HOST buffers: copies x and the logits to the device, runs the forward,
+ * copies y back and synchronises the stream before returning.  Pinned host memory makes the
+ * copies asynchronous with respect to other streams; pageable memory works too. */
+dynamo_status dynamo_moe_forward_host(dynamo_ctx* ctx, const void* x_host, const float* logits_host, int32_t T,
+                                      void* y_host, int32_t y_dtype, void* stream);
+
+/* Unpack the stored representation back to logical codes, for parity checks.
+ *   q : dev uint8 [out, in] logical codes (row-major, out = f for gate/up, d for down)
+ *   scale_f16, zero_f16 : dev uint16 [out, in/G] fp16 bit patterns
+ * which = DYNAMO_CODES_*; the HI variants exist for gate/up of routed experts with bits < 8
+ * (ERR_BITS otherwise). */
+dynamo_status dynamo_export_codes(dynamo_ctx* ctx, int32_t expert, int32_t matrix, uint8_t* q,
+                                  uint16_t* scale_f16, uint16_t* zero_f16, int32_t which, void* stream);
+
+/* Algorithmic HBM bytes of one expert as the forward streams it: packed base codes + base params
+ * of the three matrices, plus (bits < 8) the 8-bit-valued fp16 tiles of its currently significant
+ * channels.  Host only (uses the sets last installed). */
+dynamo_status dynamo_expert_stream_bytes(dynamo_ctx* ctx, int32_t expert, size_t* bytes);
+
+/* Synchronises the stream, reads the device status word: DYNAMO_OK or DYNAMO_ERR_TIMEOUT, and
+ * clears it. */
+dynamo_status dynamo_poll_status(dynamo_ctx* ctx, void* stream);
+
+/* Number of kernels the library launched through this context since creation (host counter). */
+int64_t dynamo_kernel_launches(const dynamo_ctx* ctx);
+
+const char* dynamo_status_str(dynamo_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DYNAMO_H_ */

@@ -1,0 +1,292 @@
+"""Thin ctypes binding of ``libdynamo.so`` (argument marshalling only).
+
+Module-level functions carry the C-ABI names (``dynamo_create``, ``dynamo_pack_experts``,
+``dynamo_set_channel_switch``, ``dynamo_moe_forward`` ...) and take raw pointers / sizes;
+``DynamoLayer`` wraps one context together with the torch tensors that own its device
+memory.  Every step of the path runs in the library's CUDA kernels; torch is used for
+device memory and streams only.  A missing library raises: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdynamo.so")
+_lib = None
+
+OK = 0
+BF16, F32 = 0, 1
+MAT_GATE, MAT_UP, MAT_DOWN = 0, 1, 2
+CODES_BASE, CODES_HI_POOL, CODES_HI_ACTIVE = 0, 1, 2
+SWITCH_SELECT, SWITCH_REQUANT = 0, 1
+
+STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_BITS", "ERR_ALIGN", "ERR_ARENA_TOO_SMALL", "ERR_INDEX_RANGE",
+                "ERR_INDEX_DUP", "ERR_NOT_CACHED", "ERR_STATE", "ERR_TOKENS", "ERR_CUDA", "ERR_TIMEOUT"]
+
+EXPORTED = ["dynamo_create", "dynamo_destroy", "dynamo_arena_bytes", "dynamo_pack_experts",
+            "dynamo_set_channel_switch", "dynamo_set_channel_switch_many", "dynamo_set_switch_mode",
+            "dynamo_moe_forward", "dynamo_moe_forward_host", "dynamo_export_codes", "dynamo_expert_stream_bytes",
+            "dynamo_poll_status", "dynamo_kernel_launches", "dynamo_status_str"]
+
+
+class LayerDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("d_model", "d_ff", "n_experts", "n_shared", "top_k", "group_size", "max_sig", "cache_size",
+                 "max_tokens", "renormalize")]
+
+
+class DebugOut(ctypes.Structure):
+    _fields_ = [("topk_idx", ctypes.c_void_p), ("topk_w", ctypes.c_void_p), ("expert_offsets", ctypes.c_void_p),
+                ("perm", ctypes.c_void_p)]
+
+
+class DynamoError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{where}: {name} ({status_str(status)})")
+
+
+def load():
+    """Open the library; raises if it has not been built (no CPU fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with paper_2503_21135_b200.build.build_library()")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+        i32p = ctypes.POINTER(ctypes.c_int32)
+        L.dynamo_create.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(vp)]
+        L.dynamo_destroy.argtypes = [vp]
+        L.dynamo_arena_bytes.argtypes = [ctypes.POINTER(LayerDesc), i32p, ctypes.POINTER(sz), ctypes.POINTER(sz)]
+        L.dynamo_pack_experts.argtypes = [vp, vp, vp, vp, i32p, i32p, vp, sz, vp, sz, vp]
+        L.dynamo_set_channel_switch.argtypes = [vp, i32p, i32p, vp]
+        L.dynamo_set_channel_switch_many.argtypes = [ctypes.POINTER(vp), i32, i32p, i32p, vp]
+        L.dynamo_set_switch_mode.argtypes = [vp, i32]
+        L.dynamo_moe_forward.argtypes = [vp, vp, vp, i32, vp, i32, ctypes.POINTER(DebugOut), vp]
+        L.dynamo_moe_forward_host.argtypes = [vp, vp, vp, i32, vp, i32, vp]
+        L.dynamo_export_codes.argtypes = [vp, i32, i32, vp, vp, vp, i32, vp]
+        L.dynamo_expert_stream_bytes.argtypes = [vp, i32, ctypes.POINTER(sz)]
+        L.dynamo_poll_status.argtypes = [vp, vp]
+        L.dynamo_kernel_launches.argtypes = [vp]
+        L.dynamo_kernel_launches.restype = ctypes.c_int64
+        L.dynamo_status_str.argtypes = [i32]
+        L.dynamo_status_str.restype = ctypes.c_char_p
+        for name in EXPORTED[:-2]:
+            getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def status_str(status: int) -> str:
+    return load().dynamo_status_str(int(status)).decode()
+
+
+def _i32p(a: Optional[np.ndarray]):
+    if a is None:
+        return ctypes.cast(None, ctypes.POINTER(ctypes.c_int32))
+    assert a.dtype == np.int32 and a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+
+
+# ---- C-ABI names (raw pointers and sizes) --------------------------------------------------
+
+def dynamo_create(desc: LayerDesc) -> "tuple[int, Optional[int]]":
+    h = ctypes.c_void_p()
+    st = load().dynamo_create(ctypes.byref(desc) if desc is not None else None, ctypes.byref(h))
+    return st, h.value
+
+
+def dynamo_destroy(ctx) -> int:
+    return load().dynamo_destroy(ctx)
+
+
+def dynamo_arena_bytes(desc: LayerDesc, bits: Optional[np.ndarray]):
+    wb, sb = ctypes.c_size_t(), ctypes.c_size_t()
+    st = load().dynamo_arena_bytes(ctypes.byref(desc), _i32p(bits), ctypes.byref(wb), ctypes.byref(sb))
+    return st, wb.value, sb.value
+
+
+def dynamo_pack_experts(ctx, w_gate, w_up, w_down, bits, cache_idx, arena, arena_bytes, ws, ws_bytes, stream) -> int:
+    return load().dynamo_pack_experts(ctx, w_gate, w_up, w_down, _i32p(bits), _i32p(cache_idx), arena, arena_bytes,
+                                      ws, ws_bytes, stream)
+
+
+def dynamo_set_channel_switch(ctx, sig_idx, sig_cnt, stream) -> int:
+    return load().dynamo_set_channel_switch(ctx, _i32p(sig_idx), _i32p(sig_cnt), stream)
+
+
+def dynamo_set_channel_switch_many(ctxs: Sequence[int], sig_idx, sig_cnt, stream) -> int:
+    arr = (ctypes.c_void_p * len(ctxs))(*ctxs)
+    return load().dynamo_set_channel_switch_many(arr, len(ctxs), _i32p(sig_idx), _i32p(sig_cnt), stream)
+
+
+def dynamo_set_switch_mode(ctx, mode: int) -> int:
+    return load().dynamo_set_switch_mode(ctx, mode)
+
+
+def dynamo_moe_forward(ctx, x, logits, T, y, y_dtype, dbg: Optional[DebugOut], stream) -> int:
+    return load().dynamo_moe_forward(ctx, x, logits, T, y, y_dtype, ctypes.byref(dbg) if dbg is not None else None,
+                                     stream)
+
+
+def dynamo_moe_forward_host(ctx, x_host, logits_host, T, y_host, y_dtype, stream) -> int:
+    return load().dynamo_moe_forward_host(ctx, x_host, logits_host, T, y_host, y_dtype, stream)
+
+
+def dynamo_export_codes(ctx, expert, matrix, q, scale, zero, which, stream) -> int:
+    return load().dynamo_export_codes(ctx, expert, matrix, q, scale, zero, which, stream)
+
+
+def dynamo_expert_stream_bytes(ctx, expert: int):
+    b = ctypes.c_size_t()
+    st = load().dynamo_expert_stream_bytes(ctx, expert, ctypes.byref(b))
+    return st, b.value
+
+
+def dynamo_poll_status(ctx, stream) -> int:
+    return load().dynamo_poll_status(ctx, stream)
+
+
+def dynamo_kernel_launches(ctx) -> int:
+    return int(load().dynamo_kernel_launches(ctx))
+
+
+# ---- convenience wrapper owning the torch buffers ------------------------------------------
+
+def _check(st: int, where: str) -> None:
+    if st != OK:
+        raise DynamoError(st, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+class DynamoLayer:
+    """One MoE layer context plus the torch tensors that own its arenas."""
+
+    def __init__(self, d_model, d_ff, n_experts, top_k, group_size, max_sig, cache_size, max_tokens,
+                 n_shared=0, renormalize=True, workspace: Optional[torch.Tensor] = None, device="cuda:0"):
+        self.desc = LayerDesc(d_model, d_ff, n_experts, n_shared, top_k, group_size, max_sig, cache_size, max_tokens,
+                              1 if renormalize else 0)
+        st, self.ctx = dynamo_create(self.desc)
+        _check(st, "dynamo_create")
+        self.device = torch.device(device)
+        self.arena: Optional[torch.Tensor] = None
+        self.workspace = workspace
+
+    @classmethod
+    def from_config(cls, cfg, max_tokens=None, **kw):
+        return cls(cfg.d_model, cfg.d_ff, cfg.n_experts, cfg.top_k, cfg.group_size, cfg.max_sig, cfg.cache_size,
+                   max_tokens or max(cfg.tokens), n_shared=cfg.n_shared, **kw)
+
+    def close(self):
+        if self.ctx:
+            dynamo_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def arena_bytes(self, bits: np.ndarray):
+        st, wb, sb = dynamo_arena_bytes(self.desc, np.ascontiguousarray(bits, dtype=np.int32))
+        _check(st, "dynamo_arena_bytes")
+        return wb, sb
+
+    def pack_experts(self, w_gate: torch.Tensor, w_up: torch.Tensor, w_down: torch.Tensor, bits, cache_idx):
+        bits = np.ascontiguousarray(bits, dtype=np.int32)
+        cache_idx = np.ascontiguousarray(cache_idx, dtype=np.int32)
+        wb, sb = self.arena_bytes(bits)
+        self.arena = torch.empty(wb, dtype=torch.uint8, device=self.device)
+        if self.workspace is None or self.workspace.numel() < sb:
+            self.workspace = torch.empty(sb, dtype=torch.uint8, device=self.device)
+        for w in (w_gate, w_up, w_down):
+            assert w.is_cuda and w.dtype == torch.bfloat16 and w.is_contiguous()
+        st = dynamo_pack_experts(self.ctx, w_gate.data_ptr(), w_up.data_ptr(), w_down.data_ptr(), bits, cache_idx,
+                                 self.arena.data_ptr(), self.arena.numel(), self.workspace.data_ptr(),
+                                 self.workspace.numel(), _stream())
+        _check(st, "dynamo_pack_experts")
+
+    def sig_arrays(self, sets: Sequence[np.ndarray]):
+        E, S = self.desc.n_experts, self.desc.max_sig
+        idx = np.full((E, max(S, 1)), -1, dtype=np.int32)
+        cnt = np.zeros((E,), dtype=np.int32)
+        for e, s in enumerate(sets):
+            s = np.asarray(s, dtype=np.int32)
+            cnt[e] = len(s)
+            idx[e, : min(len(s), S)] = s[:S]
+        return idx[:, :S] if S > 0 else idx[:, :0], cnt
+
+    def set_channel_switch(self, sets: Sequence[np.ndarray]):
+        idx, cnt = self.sig_arrays(sets)
+        st = dynamo_set_channel_switch(self.ctx, np.ascontiguousarray(idx), cnt, _stream())
+        _check(st, "dynamo_set_channel_switch")
+
+    def set_switch_mode(self, mode: int):
+        _check(dynamo_set_switch_mode(self.ctx, mode), "dynamo_set_switch_mode")
+
+    def forward(self, x: torch.Tensor, logits: torch.Tensor, y_dtype=F32, debug=False, y: Optional[torch.Tensor] = None):
+        T = x.shape[0]
+        assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
+        assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous()
+        if y is None:
+            y = torch.empty((T, self.desc.d_model), dtype=torch.float32 if y_dtype == F32 else torch.bfloat16,
+                            device=x.device)
+        dbg, outs = None, None
+        if debug:
+            k, E = self.desc.top_k, self.desc.n_experts
+            outs = {"idx": torch.empty((T, k), dtype=torch.int32, device=x.device),
+                    "w": torch.empty((T, k), dtype=torch.float32, device=x.device),
+                    "offsets": torch.empty((E + 1,), dtype=torch.int32, device=x.device),
+                    "perm": torch.empty((T * k,), dtype=torch.int32, device=x.device)}
+            dbg = DebugOut(outs["idx"].data_ptr(), outs["w"].data_ptr(), outs["offsets"].data_ptr(),
+                           outs["perm"].data_ptr())
+        st = dynamo_moe_forward(self.ctx, x.data_ptr(), logits.data_ptr(), T, y.data_ptr(), y_dtype, dbg, _stream())
+        _check(st, "dynamo_moe_forward")
+        return (y, outs) if debug else y
+
+    def forward_host(self, x_host: torch.Tensor, logits_host: torch.Tensor, y_host: torch.Tensor, y_dtype=F32):
+        T = x_host.shape[0]
+        st = dynamo_moe_forward_host(self.ctx, x_host.data_ptr(), logits_host.data_ptr(), T, y_host.data_ptr(),
+                                     y_dtype, _stream())
+        _check(st, "dynamo_moe_forward_host")
+        return y_host
+
+    def export_codes(self, expert: int, matrix: int, which: int = CODES_BASE):
+        d, f, G = self.desc.d_model, self.desc.d_ff, self.desc.group_size
+        N, K = (d, f) if matrix == MAT_DOWN else (f, d)
+        q = torch.empty((N, K), dtype=torch.uint8, device=self.device)
+        s = torch.empty((N, K // G), dtype=torch.int16, device=self.device)
+        m = torch.empty((N, K // G), dtype=torch.int16, device=self.device)
+        st = dynamo_export_codes(self.ctx, expert, matrix, q.data_ptr(), s.data_ptr(), m.data_ptr(), which, _stream())
+        _check(st, "dynamo_export_codes")
+        return q, s, m
+
+    def stream_bytes(self, expert: int) -> int:
+        st, b = dynamo_expert_stream_bytes(self.ctx, expert)
+        _check(st, "dynamo_expert_stream_bytes")
+        return b
+
+    def poll_status(self) -> int:
+        return dynamo_poll_status(self.ctx, _stream())
+
+    def kernel_launches(self) -> int:
+        return dynamo_kernel_launches(self.ctx)
+
+
+def set_channel_switch_many(layers: List[DynamoLayer], sets_per_layer: Sequence[Sequence[np.ndarray]]):
+    """One switch event for a stack of layers: one upload, one launch."""
+    idxs, cnts = zip(*(l.sig_arrays(s) for l, s in zip(layers, sets_per_layer)))
+    idx = np.ascontiguousarray(np.stack(idxs), dtype=np.int32)
+    cnt = np.ascontiguousarray(np.stack(cnts), dtype=np.int32)
+    st = dynamo_set_channel_switch_many([l.ctx for l in layers], idx, cnt, _stream())
+    _check(st, "dynamo_set_channel_switch_many")

@@ -1,0 +1,562 @@
+// Host side of the C-ABI: context, arena / workspace layout, argument validation, launches.
+#include <algorithm>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/dynamo.h"
+#include "common.cuh"
+
+namespace dyn {
+cudaError_t launch_pack_blocks(const void* src_a, const void* src_b, int n_rows_blocks, int K, int G, int bits,
+                               int fused, void* dst, cudaStream_t st);
+cudaError_t launch_pack_hi(const void* w_gate, const void* w_up, int f, int d, int G, int P,
+                           const int32_t* cache_idx_dev, const ExpertDev& ex, cudaStream_t st);
+cudaError_t launch_requant(const LayerDev* L, int f, const int32_t* items_dev, int n_items, cudaStream_t st);
+cudaError_t launch_export(const LayerDev* L, int e, int mat, int which, long long n_elems, uint8_t* q, uint16_t* sc,
+                          uint16_t* zr, cudaStream_t st);
+cudaError_t launch_route(const float* logits, int T, int E, int k, int renorm, int32_t* idx, float* w,
+                         cudaStream_t st);
+cudaError_t launch_scan(const WsDev& ws, int E, int Es, int k, cudaStream_t st);
+cudaError_t launch_gather(const LayerDev* L, const WsDev& ws, const void* x, cudaStream_t st);
+cudaError_t launch_combine(const WsDev& ws, int d, int k, int Es, void* y, int y_f32, long long split_stride,
+                           cudaStream_t st);
+cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, int nt8, int n_tc, int n_rb, int ksplit,
+                              int n_experts, long long split_stride, int smem_bytes, cudaStream_t st);
+cudaError_t launch_switch(const SwitchLayers& layers, int n_layers, int E, const int32_t* staging, int per_layer_ints,
+                          cudaStream_t st);
+}  // namespace dyn
+
+using namespace dyn;
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+constexpr int ROW_PAD = 32;            // extra activation rows so a token chunk may read past the last row
+constexpr int MAX_SWITCH_LAYERS = 64;
+constexpr int FFN_SMEM_BYTES = 110 * 1024;
+constexpr int DECODE_ROWS = 1024;      // up to this many permuted rows the down GEMM is split along K
+constexpr int MAX_KSPLIT = 8;
+
+inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
+
+struct ArenaLayout {
+    size_t header = 0;
+    std::vector<size_t> w13, w2, s8m8_g, s8m8_u, q8_g, q8_u, cw_g, cw_u, pool_hi;
+    size_t cache_idx = 0, sig_chan = 0, sig_pool = 0, sig_cnt = 0, sigmask = 0;
+    size_t total = 0;
+};
+
+struct WsLayout {
+    size_t status, counts, offsets, topk_idx, topk_w, perm, pos, row_token, row_expert, xperm, xsig, hbuf, ypart,
+        stage_x, stage_logits, stage_y, stage_switch, total;
+    long long ypart_rows;  // capacity in rows of one K split
+};
+
+inline int s_pad_of(const dynamo_layer_desc& D) { return (D.max_sig + 15) / 16 * 16; }
+inline int ksplit_for(const dynamo_layer_desc& D, int T) {
+    const long long R = (long long)T * (D.top_k + D.n_shared);
+    return R <= DECODE_ROWS ? std::min(MAX_KSPLIT, D.d_ff / KC) : 1;
+}
+inline int switch_ints_per_layer(const dynamo_layer_desc& D) { return D.n_experts * (2 * s_pad_of(D) + 1); }
+
+dynamo_status check_desc(const dynamo_layer_desc* D) {
+    if (!D) return DYNAMO_ERR_NULL;
+    if (D->d_model <= 0 || D->d_ff <= 0 || D->d_model % 256 || D->d_ff % 128) return DYNAMO_ERR_SHAPE;
+    if (D->group_size != 64 && D->group_size != 128) return DYNAMO_ERR_SHAPE;
+    if (D->n_experts < 1 || D->n_experts > 256 || D->n_shared < 0 || D->n_experts + D->n_shared > MAX_EXPERTS)
+        return DYNAMO_ERR_SHAPE;
+    if (D->top_k < 1 || D->top_k > 8 || D->top_k > D->n_experts) return DYNAMO_ERR_SHAPE;
+    if (D->max_sig < 0 || D->max_sig > 256 || D->cache_size < D->max_sig || D->cache_size > D->d_model ||
+        D->cache_size > 65535)
+        return DYNAMO_ERR_SHAPE;
+    if (D->max_tokens < 1 || (long long)D->max_tokens * (D->top_k + D->n_shared) > (1ll << 24)) return DYNAMO_ERR_SHAPE;
+    return DYNAMO_OK;
+}
+
+dynamo_status check_bits(const dynamo_layer_desc& D, const int32_t* bits) {
+    if (!bits) return DYNAMO_ERR_NULL;
+    for (int e = 0; e < D.n_experts + D.n_shared; ++e) {
+        const int b = bits[e];
+        if (e >= D.n_experts) {
+            if (b != 8) return DYNAMO_ERR_BITS;
+        } else if (b != 2 && b != 3 && b != 4 && b != 8) {
+            return DYNAMO_ERR_BITS;
+        }
+    }
+    return DYNAMO_OK;
+}
+
+void arena_layout(const dynamo_layer_desc& D, const int32_t* bits, ArenaLayout& A) {
+    const int n = D.n_experts + D.n_shared;
+    const size_t d = D.d_model, f = D.d_ff, G = D.group_size, P = D.cache_size;
+    const size_t n_rb13 = 2 * f / RB, n_kc13 = d / KC, n_rb2 = d / RB, n_kc2 = f / KC;
+    size_t off = align_up(sizeof(LayerDev));
+    A.header = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    A.w13.assign(n, 0); A.w2.assign(n, 0);
+    A.s8m8_g.assign(n, 0); A.s8m8_u.assign(n, 0); A.q8_g.assign(n, 0); A.q8_u.assign(n, 0);
+    A.cw_g.assign(n, 0); A.cw_u.assign(n, 0); A.pool_hi.assign(n, 0);
+    for (int e = 0; e < n; ++e) {
+        const size_t blk = block_bytes(bits[e], (int)G);
+        A.w13[e] = take(n_rb13 * n_kc13 * blk);
+        A.w2[e] = take(n_rb2 * n_kc2 * blk);
+    }
+    for (int e = 0; e < D.n_experts; ++e) {
+        if (bits[e] >= HI_BITS) continue;
+        A.s8m8_g[e] = take(f * (d / G) * 4);
+        A.s8m8_u[e] = take(f * (d / G) * 4);
+        A.q8_g[e] = take(P * f);
+        A.q8_u[e] = take(P * f);
+        A.cw_g[e] = take(P * f * 2);
+        A.cw_u[e] = take(P * f * 2);
+        A.pool_hi[e] = take(n_rb13 * (P + 1) * RB * 2);
+    }
+    const size_t S_pad = s_pad_of(D);
+    A.cache_idx = take((size_t)D.n_experts * P * 4);
+    A.sig_chan = take((size_t)D.n_experts * S_pad * 4);
+    A.sig_pool = take((size_t)D.n_experts * S_pad * 4);
+    A.sig_cnt = take((size_t)D.n_experts * 4);
+    A.sigmask = take((size_t)D.n_experts * (d / 32) * 4);
+    A.total = off;
+}
+
+void ws_layout(const dynamo_layer_desc& D, WsLayout& W) {
+    const size_t n = D.n_experts + D.n_shared, T = D.max_tokens, k = D.top_k, kk = D.top_k + D.n_shared;
+    const size_t R = T * kk, d = D.d_model, f = D.d_ff, S_pad = s_pad_of(D);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    W.status = take(256);
+    W.counts = take(n * 4);
+    W.offsets = take((n + 1) * 4);
+    W.topk_idx = take(T * k * 4);
+    W.topk_w = take(T * k * 4);
+    W.perm = take(T * k * 4);
+    W.pos = take(T * kk * 4);
+    W.row_token = take(R * 4);
+    W.row_expert = take(R * 4);
+    W.xperm = take((R + ROW_PAD) * (d / KC) * XROW);
+    W.xsig = take((R + ROW_PAD) * std::max<size_t>(S_pad, 16) * 2);
+    W.hbuf = take((R + ROW_PAD) * (f / KC) * XROW);
+    const size_t ks = std::min<size_t>(MAX_KSPLIT, f / KC);
+    const size_t small_rows = std::min<size_t>(R, DECODE_ROWS);
+    W.ypart_rows = (long long)std::max(R, small_rows);
+    W.ypart = take(std::max(R, ks * small_rows) * d * 4);
+    W.stage_x = take(T * d * 2);
+    W.stage_logits = take(T * (size_t)D.n_experts * 4);
+    W.stage_y = take(T * d * 4);
+    W.stage_switch = take((size_t)MAX_SWITCH_LAYERS * (switch_ints_per_layer(D) + (size_t)D.n_experts * S_pad) * 4);
+    W.total = off;
+}
+
+}  // namespace
+
+struct dynamo_ctx {
+    dynamo_layer_desc D;
+    bool packed = false;
+    std::vector<int32_t> bits;
+    std::vector<int32_t> cache_idx;              // host copy [E][P]
+    std::vector<std::vector<int32_t>> sig;       // current sets, in slot order
+    ArenaLayout A;
+    WsLayout W;
+    uint8_t* arena = nullptr;
+    uint8_t* ws = nullptr;
+    LayerDev host_layer;                         // host mirror of the arena header
+    int switch_mode = DYNAMO_SWITCH_SELECT;
+    int64_t launches = 0;
+    std::vector<int32_t> upload;                 // scratch for switch uploads
+};
+
+namespace {
+
+WsDev make_ws(const dynamo_ctx* c, int T) {
+    const dynamo_layer_desc& D = c->D;
+    WsDev w;
+    uint8_t* b = c->ws;
+    w.counts = (int32_t*)(b + c->W.counts);
+    w.offsets = (int32_t*)(b + c->W.offsets);
+    w.topk_idx = (int32_t*)(b + c->W.topk_idx);
+    w.topk_w = (float*)(b + c->W.topk_w);
+    w.perm = (int32_t*)(b + c->W.perm);
+    w.pos = (int32_t*)(b + c->W.pos);
+    w.row_token = (int32_t*)(b + c->W.row_token);
+    w.row_expert = (int32_t*)(b + c->W.row_expert);
+    w.xperm = b + c->W.xperm;
+    w.xsig = (__half*)(b + c->W.xsig);
+    w.hbuf = b + c->W.hbuf;
+    w.ypart = (float*)(b + c->W.ypart);
+    w.status = (int32_t*)(b + c->W.status);
+    w.T = T;
+    w.R = T * (D.top_k + D.n_shared);
+    w.ksplit = ksplit_for(D, T);
+    w.pad_ = 0;
+    return w;
+}
+
+#define CUDA_TRY(expr)                                  \
+    do {                                                \
+        cudaError_t err__ = (expr);                     \
+        if (err__ != cudaSuccess) return DYNAMO_ERR_CUDA; \
+    } while (0)
+
+// Validate one layer's new sets against its cache; on success fill `lists` (slot order = caller order).
+dynamo_status validate_sets(const dynamo_ctx* c, const int32_t* sig_idx, const int32_t* sig_cnt,
+                            std::vector<std::vector<int32_t>>& lists) {
+    const dynamo_layer_desc& D = c->D;
+    lists.assign(D.n_experts, {});
+    std::vector<uint8_t> seen(D.d_model);
+    for (int e = 0; e < D.n_experts; ++e) {
+        const int cnt = sig_cnt[e];
+        if (cnt < 0 || cnt > D.max_sig) return DYNAMO_ERR_INDEX_RANGE;
+        std::fill(seen.begin(), seen.end(), 0);
+        const int32_t* ci = c->cache_idx.data() + (size_t)e * D.cache_size;
+        for (int j = 0; j < cnt; ++j) {
+            const int ch = sig_idx[(size_t)e * D.max_sig + j];
+            if (ch < 0 || ch >= D.d_model) return DYNAMO_ERR_INDEX_RANGE;
+            if (seen[ch]) return DYNAMO_ERR_INDEX_DUP;
+            seen[ch] = 1;
+            if (!std::binary_search(ci, ci + D.cache_size, ch)) return DYNAMO_ERR_NOT_CACHED;
+            lists[e].push_back(ch);
+        }
+    }
+    return DYNAMO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* dynamo_status_str(dynamo_status s) {
+    switch (s) {
+        case DYNAMO_OK: return "ok";
+        case DYNAMO_ERR_NULL: return "null pointer";
+        case DYNAMO_ERR_SHAPE: return "unsupported shape";
+        case DYNAMO_ERR_BITS: return "unsupported bit-width";
+        case DYNAMO_ERR_ALIGN: return "buffer not 256-byte aligned";
+        case DYNAMO_ERR_ARENA_TOO_SMALL: return "arena or workspace too small";
+        case DYNAMO_ERR_INDEX_RANGE: return "channel index or count out of range";
+        case DYNAMO_ERR_INDEX_DUP: return "duplicate or unsorted channel index";
+        case DYNAMO_ERR_NOT_CACHED: return "channel not in the expert's channel cache";
+        case DYNAMO_ERR_STATE: return "experts not packed yet";
+        case DYNAMO_ERR_TOKENS: return "token count out of range";
+        case DYNAMO_ERR_CUDA: return "CUDA runtime error";
+        case DYNAMO_ERR_TIMEOUT: return "device-side wait expired";
+    }
+    return "unknown status";
+}
+
+dynamo_status dynamo_create(const dynamo_layer_desc* desc, dynamo_ctx** out) {
+    if (!out) return DYNAMO_ERR_NULL;
+    *out = nullptr;
+    dynamo_status st = check_desc(desc);
+    if (st != DYNAMO_OK) return st;
+    dynamo_ctx* c = new (std::nothrow) dynamo_ctx();
+    if (!c) return DYNAMO_ERR_NULL;
+    c->D = *desc;
+    c->D.renormalize = desc->renormalize ? 1 : 0;
+    ws_layout(c->D, c->W);
+    *out = c;
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_destroy(dynamo_ctx* ctx) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    delete ctx;
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_arena_bytes(const dynamo_layer_desc* desc, const int32_t* bits, size_t* weights_bytes,
+                                 size_t* workspace_bytes) {
+    dynamo_status st = check_desc(desc);
+    if (st != DYNAMO_OK) return st;
+    if (!weights_bytes || !workspace_bytes) return DYNAMO_ERR_NULL;
+    st = check_bits(*desc, bits);
+    if (st != DYNAMO_OK) return st;
+    ArenaLayout A;
+    arena_layout(*desc, bits, A);
+    WsLayout W;
+    ws_layout(*desc, W);
+    *weights_bytes = A.total;
+    *workspace_bytes = W.total;
+    return DYNAMO_OK;
+}
+
+int64_t dynamo_kernel_launches(const dynamo_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+dynamo_status dynamo_set_switch_mode(dynamo_ctx* ctx, int32_t mode) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    if (mode != DYNAMO_SWITCH_SELECT && mode != DYNAMO_SWITCH_REQUANT) return DYNAMO_ERR_SHAPE;
+    ctx->switch_mode = mode;
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_pack_experts(dynamo_ctx* ctx, const void* w_gate, const void* w_up, const void* w_down,
+                                  const int32_t* bits, const int32_t* cache_idx, void* weights_arena,
+                                  size_t weights_bytes, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!ctx || !w_gate || !w_up || !w_down || !bits || !weights_arena || !workspace) return DYNAMO_ERR_NULL;
+    const dynamo_layer_desc& D = ctx->D;
+    if (D.cache_size > 0 && !cache_idx) return DYNAMO_ERR_NULL;
+    dynamo_status stt = check_bits(D, bits);
+    if (stt != DYNAMO_OK) return stt;
+    for (int e = 0; e < D.n_experts; ++e)
+        for (int p = 0; p < D.cache_size; ++p) {
+            const int c = cache_idx[(size_t)e * D.cache_size + p];
+            if (c < 0 || c >= D.d_model) return DYNAMO_ERR_INDEX_RANGE;
+            if (p > 0 && c <= cache_idx[(size_t)e * D.cache_size + p - 1]) return DYNAMO_ERR_INDEX_DUP;
+        }
+    if (((uintptr_t)weights_arena % ALIGN) || ((uintptr_t)workspace % ALIGN)) return DYNAMO_ERR_ALIGN;
+    ArenaLayout A;
+    arena_layout(D, bits, A);
+    if (weights_bytes < A.total || workspace_bytes < ctx->W.total) return DYNAMO_ERR_ARENA_TOO_SMALL;
+
+    cudaStream_t st = (cudaStream_t)stream;
+    const int n = D.n_experts + D.n_shared;
+    const int d = D.d_model, f = D.d_ff, G = D.group_size, P = D.cache_size;
+    ctx->packed = false;
+    ctx->A = A;
+    ctx->arena = (uint8_t*)weights_arena;
+    ctx->ws = (uint8_t*)workspace;
+    ctx->bits.assign(bits, bits + n);
+    ctx->cache_idx.assign(cache_idx, cache_idx + (size_t)D.n_experts * P);
+    ctx->sig.assign(D.n_experts, {});
+
+    CUDA_TRY(cudaMemsetAsync(ctx->arena, 0, A.total, st));
+    CUDA_TRY(cudaMemsetAsync(ctx->ws, 0, ctx->W.total, st));
+
+    LayerDev& L = ctx->host_layer;
+    std::memset(&L, 0, sizeof(L));
+    L.d = d; L.f = f; L.E = D.n_experts; L.Es = D.n_shared; L.k = D.top_k; L.G = G;
+    L.S = D.max_sig; L.S_pad = s_pad_of(D); L.P = P; L.renorm = D.renormalize;
+    L.n_rb13 = 2 * f / RB; L.n_kc13 = d / KC; L.n_rb2 = d / RB; L.n_kc2 = f / KC;
+    uint8_t* base = ctx->arena;
+    L.cache_idx = (int32_t*)(base + A.cache_idx);
+    L.sig_chan = (int32_t*)(base + A.sig_chan);
+    L.sig_pool = (int32_t*)(base + A.sig_pool);
+    L.sig_cnt = (int32_t*)(base + A.sig_cnt);
+    L.sigmask = (uint32_t*)(base + A.sigmask);
+    std::vector<int> order(n);
+    for (int e = 0; e < n; ++e) order[e] = e;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return bits[a] > bits[b]; });
+    for (int e = 0; e < n; ++e) L.order[e] = order[e];
+    for (int e = 0; e < n; ++e) {
+        ExpertDev& x = L.ex[e];
+        x.bits = bits[e];
+        x.blk_bytes = block_bytes(bits[e], G);
+        x.w13 = base + A.w13[e];
+        x.w2 = base + A.w2[e];
+        x.switchable = (e < D.n_experts && bits[e] < HI_BITS) ? 1 : 0;
+        if (x.switchable) {
+            x.s8m8[0] = (uint32_t*)(base + A.s8m8_g[e]);
+            x.s8m8[1] = (uint32_t*)(base + A.s8m8_u[e]);
+            x.pool_q8[0] = base + A.q8_g[e];
+            x.pool_q8[1] = base + A.q8_u[e];
+            x.cache_w[0] = (__nv_bfloat16*)(base + A.cw_g[e]);
+            x.cache_w[1] = (__nv_bfloat16*)(base + A.cw_u[e]);
+            x.pool_hi = (__half*)(base + A.pool_hi[e]);
+        }
+    }
+    CUDA_TRY(cudaMemcpyAsync(base, &L, sizeof(L), cudaMemcpyHostToDevice, st));
+    if (P > 0)
+        CUDA_TRY(cudaMemcpyAsync(L.cache_idx, ctx->cache_idx.data(), ctx->cache_idx.size() * 4, cudaMemcpyHostToDevice,
+                                 st));
+
+    const __nv_bfloat16* wg = (const __nv_bfloat16*)w_gate;
+    const __nv_bfloat16* wu = (const __nv_bfloat16*)w_up;
+    const __nv_bfloat16* wd = (const __nv_bfloat16*)w_down;
+    for (int e = 0; e < n; ++e) {
+        const size_t eo = (size_t)e * f * d;
+        CUDA_TRY(launch_pack_blocks(wg + eo, wu + eo, L.n_rb13, d, G, bits[e], 1, (void*)L.ex[e].w13, st));
+        CUDA_TRY(launch_pack_blocks(wd + eo, nullptr, L.n_rb2, f, G, bits[e], 0, (void*)L.ex[e].w2, st));
+        ctx->launches += 2;
+        if (L.ex[e].switchable && P > 0) {
+            CUDA_TRY(launch_pack_hi(wg + eo, wu + eo, f, d, G, P, L.cache_idx + (size_t)e * P, L.ex[e], st));
+            ctx->launches += 1;
+        }
+    }
+    ctx->packed = true;
+    // install the empty significant sets (sig_pool -> zero tile, sig_chan -> -1)
+    std::vector<int32_t> zero_cnt(D.n_experts, 0);
+    std::vector<int32_t> dummy((size_t)D.n_experts * std::max(1, D.max_sig), 0);
+    dynamo_status s2 = dynamo_set_channel_switch(ctx, dummy.data(), zero_cnt.data(), stream);
+    if (s2 != DYNAMO_OK) ctx->packed = false;
+    return s2;
+}
+
+dynamo_status dynamo_set_channel_switch_many(dynamo_ctx* const* ctxs, int32_t n_layers, const int32_t* sig_idx,
+                                             const int32_t* sig_cnt, void* stream) {
+    if (!ctxs || !sig_idx || !sig_cnt) return DYNAMO_ERR_NULL;
+    if (n_layers < 1 || n_layers > MAX_SWITCH_LAYERS) return DYNAMO_ERR_SHAPE;
+    for (int l = 0; l < n_layers; ++l) {
+        if (!ctxs[l]) return DYNAMO_ERR_NULL;
+        if (!ctxs[l]->packed) return DYNAMO_ERR_STATE;
+        if (std::memcmp(&ctxs[l]->D, &ctxs[0]->D, sizeof(dynamo_layer_desc)) != 0) return DYNAMO_ERR_SHAPE;
+    }
+    dynamo_ctx* c0 = ctxs[0];
+    const dynamo_layer_desc& D = c0->D;
+    const int E = D.n_experts, S = D.max_sig, S_pad = s_pad_of(D), P = D.cache_size;
+    const int per_layer = switch_ints_per_layer(D);
+    // validate everything first: all-or-nothing
+    std::vector<std::vector<std::vector<int32_t>>> lists(n_layers);
+    for (int l = 0; l < n_layers; ++l) {
+        dynamo_status st = validate_sets(ctxs[l], sig_idx + (size_t)l * E * S, sig_cnt + (size_t)l * E, lists[l]);
+        if (st != DYNAMO_OK) return st;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    std::vector<int32_t>& up = c0->upload;
+    up.assign((size_t)n_layers * per_layer, 0);
+    SwitchLayers layers;
+    std::memset(&layers, 0, sizeof(layers));
+    int32_t* staging = (int32_t*)(c0->ws + c0->W.stage_switch);
+    int32_t* items_dev = staging + (size_t)MAX_SWITCH_LAYERS * per_layer;
+    for (int l = 0; l < n_layers; ++l) {
+        dynamo_ctx* c = ctxs[l];
+        layers.layer[l] = (const LayerDev*)c->arena;
+        int32_t* chan = up.data() + (size_t)l * per_layer;
+        int32_t* pool = chan + (size_t)E * S_pad;
+        int32_t* cnt = pool + (size_t)E * S_pad;
+        std::vector<int32_t> items;  // entering cached channels (expert << 16 | pool position)
+        for (int e = 0; e < E; ++e) {
+            const int32_t* ci = c->cache_idx.data() + (size_t)e * P;
+            const bool sw = c->bits[e] < HI_BITS;
+            const std::vector<int32_t>& lst = lists[l][e];
+            cnt[e] = sw ? (int32_t)lst.size() : 0;
+            for (int j = 0; j < S_pad; ++j) {
+                chan[e * S_pad + j] = -1;
+                pool[e * S_pad + j] = P;
+            }
+            if (!sw) continue;
+            for (size_t j = 0; j < lst.size(); ++j) {
+                const int p = (int)(std::lower_bound(ci, ci + P, lst[j]) - ci);
+                chan[e * S_pad + j] = lst[j];
+                pool[e * S_pad + j] = p;
+                if (c->switch_mode == DYNAMO_SWITCH_REQUANT &&
+                    std::find(c->sig[e].begin(), c->sig[e].end(), lst[j]) == c->sig[e].end())
+                    items.push_back((e << 16) | p);
+            }
+        }
+        if (!items.empty()) {
+            // channel replacement + requantization of the entering channels from the bf16 cache
+            int32_t* dst = items_dev + (size_t)l * E * S_pad;
+            CUDA_TRY(cudaMemcpyAsync(dst, items.data(), items.size() * 4, cudaMemcpyHostToDevice, st));
+            CUDA_TRY(launch_requant(layers.layer[l], D.d_ff, dst, (int)items.size(), st));
+            c->launches += 1;
+        }
+    }
+    CUDA_TRY(cudaMemcpyAsync(staging, up.data(), up.size() * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(launch_switch(layers, n_layers, E, staging, per_layer, st));
+    c0->launches += 1;
+    for (int l = 0; l < n_layers; ++l) ctxs[l]->sig = lists[l];
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_set_channel_switch(dynamo_ctx* ctx, const int32_t* sig_idx, const int32_t* sig_cnt,
+                                        void* stream) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    dynamo_ctx* one[1] = {ctx};
+    return dynamo_set_channel_switch_many(one, 1, sig_idx, sig_cnt, stream);
+}
+
+dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* router_logits, int32_t T, void* y,
+                                 int32_t y_dtype, const dynamo_debug_out* dbg, void* stream) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    if (!ctx->packed) return DYNAMO_ERR_STATE;
+    const dynamo_layer_desc& D = ctx->D;
+    if (T < 0 || T > D.max_tokens) return DYNAMO_ERR_TOKENS;
+    if (y_dtype != DYNAMO_BF16 && y_dtype != DYNAMO_F32) return DYNAMO_ERR_SHAPE;
+    if (T == 0) return DYNAMO_OK;
+    if (!x || !router_logits || !y) return DYNAMO_ERR_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    const LayerDev* L = (const LayerDev*)ctx->arena;
+    WsDev ws = make_ws(ctx, T);
+    const int n = D.n_experts + D.n_shared;
+
+    CUDA_TRY(launch_route(router_logits, T, D.n_experts, D.top_k, D.renormalize, ws.topk_idx, ws.topk_w, st));
+    CUDA_TRY(launch_scan(ws, D.n_experts, D.n_shared, D.top_k, st));
+    CUDA_TRY(launch_gather(L, ws, x, st));
+    const int nt8 = T <= 8 ? 1 : (T <= 16 ? 2 : 4);
+    const int n_tc = (T + nt8 * 8 - 1) / (nt8 * 8);
+    const long long split_stride = (long long)ws.R * D.d_model;  // partials of one K split: [R][d]
+    CUDA_TRY(launch_ffn_stream(L, ws, 1, nt8, n_tc, ctx->host_layer.n_rb13, 1, n, split_stride, FFN_SMEM_BYTES, st));
+    CUDA_TRY(launch_ffn_stream(L, ws, 0, nt8, n_tc, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, FFN_SMEM_BYTES,
+                               st));
+    CUDA_TRY(launch_combine(ws, D.d_model, D.top_k, D.n_shared, y, y_dtype == DYNAMO_F32, split_stride, st));
+    ctx->launches += 6;
+    if (dbg) {
+        const size_t tk = (size_t)T * D.top_k;
+        if (dbg->topk_idx) CUDA_TRY(cudaMemcpyAsync(dbg->topk_idx, ws.topk_idx, tk * 4, cudaMemcpyDeviceToDevice, st));
+        if (dbg->topk_w) CUDA_TRY(cudaMemcpyAsync(dbg->topk_w, ws.topk_w, tk * 4, cudaMemcpyDeviceToDevice, st));
+        if (dbg->expert_offsets)
+            CUDA_TRY(cudaMemcpyAsync(dbg->expert_offsets, ws.offsets, (size_t)(D.n_experts + 1) * 4,
+                                     cudaMemcpyDeviceToDevice, st));
+        if (dbg->perm) CUDA_TRY(cudaMemcpyAsync(dbg->perm, ws.perm, tk * 4, cudaMemcpyDeviceToDevice, st));
+    }
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_moe_forward_host(dynamo_ctx* ctx, const void* x_host, const float* logits_host, int32_t T,
+                                      void* y_host, int32_t y_dtype, void* stream) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    if (!ctx->packed) return DYNAMO_ERR_STATE;
+    const dynamo_layer_desc& D = ctx->D;
+    if (T < 0 || T > D.max_tokens) return DYNAMO_ERR_TOKENS;
+    if (y_dtype != DYNAMO_BF16 && y_dtype != DYNAMO_F32) return DYNAMO_ERR_SHAPE;
+    if (T == 0) return DYNAMO_OK;
+    if (!x_host || !logits_host || !y_host) return DYNAMO_ERR_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    void* xd = ctx->ws + ctx->W.stage_x;
+    float* ld = (float*)(ctx->ws + ctx->W.stage_logits);
+    void* yd = ctx->ws + ctx->W.stage_y;
+    CUDA_TRY(cudaMemcpyAsync(xd, x_host, (size_t)T * D.d_model * 2, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(ld, logits_host, (size_t)T * D.n_experts * 4, cudaMemcpyHostToDevice, st));
+    dynamo_status s = dynamo_moe_forward(ctx, xd, ld, T, yd, y_dtype, nullptr, stream);
+    if (s != DYNAMO_OK) return s;
+    const size_t ybytes = (size_t)T * D.d_model * (y_dtype == DYNAMO_F32 ? 4 : 2);
+    CUDA_TRY(cudaMemcpyAsync(y_host, yd, ybytes, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_export_codes(dynamo_ctx* ctx, int32_t expert, int32_t matrix, uint8_t* q, uint16_t* scale_f16,
+                                  uint16_t* zero_f16, int32_t which, void* stream) {
+    if (!ctx || !q || !scale_f16 || !zero_f16) return DYNAMO_ERR_NULL;
+    if (!ctx->packed) return DYNAMO_ERR_STATE;
+    const dynamo_layer_desc& D = ctx->D;
+    if (expert < 0 || expert >= D.n_experts + D.n_shared || matrix < 0 || matrix > 2 || which < 0 || which > 2)
+        return DYNAMO_ERR_SHAPE;
+    if (which != DYNAMO_CODES_BASE && (matrix == DYNAMO_MAT_DOWN || !ctx->host_layer.ex[expert].switchable))
+        return DYNAMO_ERR_BITS;
+    const long long n_elems = (long long)D.d_model * D.d_ff;
+    CUDA_TRY(launch_export((const LayerDev*)ctx->arena, expert, matrix, which, n_elems, q, scale_f16, zero_f16,
+                           (cudaStream_t)stream));
+    ctx->launches += 1;
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_expert_stream_bytes(dynamo_ctx* ctx, int32_t expert, size_t* bytes) {
+    if (!ctx || !bytes) return DYNAMO_ERR_NULL;
+    if (!ctx->packed) return DYNAMO_ERR_STATE;
+    const dynamo_layer_desc& D = ctx->D;
+    if (expert < 0 || expert >= D.n_experts + D.n_shared) return DYNAMO_ERR_SHAPE;
+    const size_t d = D.d_model, f = D.d_ff;
+    const size_t blocks = (2 * f / RB) * (d / KC) + (d / RB) * (f / KC);
+    size_t b = blocks * (size_t)block_bytes(ctx->bits[expert], D.group_size);
+    if (expert < D.n_experts && ctx->bits[expert] < HI_BITS) b += 2 * f * ctx->sig[expert].size() * 2;
+    *bytes = b;
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_poll_status(dynamo_ctx* ctx, void* stream) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    if (!ctx->packed) return DYNAMO_ERR_STATE;
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t word = 0;
+    CUDA_TRY(cudaMemcpyAsync(&word, ctx->ws + ctx->W.status, 4, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    if (word != STATUS_OK) {
+        CUDA_TRY(cudaMemsetAsync(ctx->ws + ctx->W.status, 0, 4, st));
+        return DYNAMO_ERR_TIMEOUT;
+    }
+    return DYNAMO_OK;
+}
+
+}  // extern "C"

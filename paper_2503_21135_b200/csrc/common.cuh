@@ -1,0 +1,170 @@
+// Shared device-side declarations of the DynaMo B200 library: arena descriptors, constants,
+// small PTX wrappers (mbarrier, bulk async copy, bounded waits).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace dyn {
+
+constexpr int RB = 256;          // weight rows per packed block
+constexpr int KC = 128;          // input indices (k) per packed block
+constexpr int ATOM_ROWS = 16;    // rows of one MMA fragment tile; a block has 16 atoms
+constexpr int XROW = 288;        // bytes per (token row, k-chunk) in activation buffers:
+                                 // 128 fp16 + two fp32 sums (k 0..63, 64..127) + pad; 288/4 = 72 = 8 (mod 32) banks
+constexpr int XROW_SUM_OFF = 256;
+constexpr int POOL_TILE_BYTES = 512;   // one cached channel's 8-bit-valued fp16 column for the 256 rows of a block
+constexpr int MAX_EXPERTS = 264;
+constexpr int HI_BITS = 8;
+
+enum : int { STATUS_OK = 0, STATUS_TIMEOUT = 1 };
+
+struct ExpertDev {
+    const uint8_t* w13;        // packed blocks of the fused gate/up matrix: [n_rb13][n_kc13][blk_bytes]
+    const uint8_t* w2;         // packed blocks of the down matrix:          [n_rb2][n_kc2][blk_bytes]
+    __half* pool_hi;           // [n_rb13][P + 1][256] fp16, value s8*q8+m8 of cached channel p (tile P = zeros)
+    uint32_t* s8m8[2];         // gate, up: [f][d/G] half2 {scale, zero} of the 8-bit quantization
+    uint8_t* pool_q8[2];       // gate, up: [P][f] 8-bit codes of the cached channels
+    __nv_bfloat16* cache_w[2]; // gate, up: [P][f] bf16 originals of the cached channels (the channel cache)
+    int32_t bits;
+    int32_t blk_bytes;         // bytes of one packed block (codes + params)
+    int32_t switchable;        // routed expert with bits < 8
+    int32_t pad_;
+};
+
+struct LayerDev {
+    int32_t d, f, E, Es, k, G, S, S_pad, P, renorm;
+    int32_t n_rb13, n_kc13, n_rb2, n_kc2;
+    int32_t* cache_idx;   // [E][P] sorted channel indices (cache headers)
+    int32_t* sig_chan;    // [E][S_pad] channel of each active slot, -1 = empty
+    int32_t* sig_pool;    // [E][S_pad] pool position of each active slot, P = zero tile
+    int32_t* sig_cnt;     // [E]
+    uint32_t* sigmask;    // [E][d/32] bit c set <=> channel c significant
+    int32_t order[MAX_EXPERTS];  // expert ids sorted by descending bits (heaviest work first)
+    ExpertDev ex[MAX_EXPERTS];
+};
+
+// Workspace pointers of one forward (passed to kernels by value).
+struct WsDev {
+    int32_t* counts;      // [E_tot]
+    int32_t* offsets;     // [E_tot + 1]
+    int32_t* topk_idx;    // [T, k]
+    float* topk_w;        // [T, k]
+    int32_t* perm;        // [T*k]
+    int32_t* pos;         // [T, k+Es]  sorted row of pair (t, j)
+    int32_t* row_token;   // [R]
+    int32_t* row_expert;  // [R]
+    uint8_t* xperm;       // [R + pad][d/128][XROW]
+    __half* xsig;         // [R + pad][S_pad]
+    uint8_t* hbuf;        // [R + pad][f/128][XROW]
+    float* ypart;         // [ksplit][R][d]
+    int32_t* status;      // device status word
+    int32_t T, R, ksplit, pad_;
+};
+
+// Layers of one switch event (kernel parameter).
+struct SwitchLayers {
+    const LayerDev* layer[64];
+};
+
+// ---- PTX helpers -----------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait: spins on the barrier phase for at most ~1 s.  On expiry (or when another thread of
+// the CTA already gave up) it records STATUS_TIMEOUT, raises the CTA-wide poison flag and returns
+// false; callers then leave their loops.
+constexpr unsigned long long WAIT_LIMIT_NS = 1000ull * 1000ull * 1000ull;
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* poison,
+                                                  int32_t* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    uint32_t spins = 0;
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 0xff) == 0) {
+            if (*poison) return false;
+            if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+                *poison = 1;
+                atomicExch(status, STATUS_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+// 1-D bulk async copy global -> shared, completion counted on an mbarrier (bytes % 16 == 0,
+// both addresses 16-byte aligned).
+__device__ __forceinline__ void bulk_g2s(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            smem_u32(smem_dst)),
+        "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// m16n8k16 fp16 x fp16 -> fp32
+__device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// ---- packed-block geometry ---------------------------------------------------------------
+
+__host__ __device__ __forceinline__ int atom_bytes(int bits) { return 256 * bits; }  // 16 rows x 128 k
+__host__ __device__ __forceinline__ int block_code_bytes(int bits) { return 4096 * bits; }
+__host__ __device__ __forceinline__ int block_bytes(int bits, int G) { return 4096 * bits + RB * (KC / G) * 4; }
+
+// Row of the fused gate/up matrix: block rb, atom a, row ra (0..15): rows 0..7 of an atom are gate
+// rows, rows 8..15 the up rows of the same eight hidden indices h = 128*rb + 8*a + (ra & 7).
+__host__ __device__ __forceinline__ int w13_hidden_index(int rb, int r) {
+    return 128 * rb + 8 * (r >> 4) + (r & 7);
+}
+__host__ __device__ __forceinline__ int w13_row_in_block(int h, int is_up) {
+    return 16 * ((h & 127) >> 3) + (h & 7) + (is_up ? 8 : 0);
+}
+
+}  // namespace dyn
