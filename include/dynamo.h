@@ -176,6 +176,29 @@ int64_t dynamo_kernel_launches(const dynamo_ctx* ctx);
 
 const char* dynamo_status_str(dynamo_status s);
 
+/* Routing + permutation for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; the step itself is the Top-K selection and one-to-many dispatch of Section II-A.)
+ * Some users of this library are not allowed to call cudaMalloc: code that runs while a CUDA graph
+ * is being captured, plugins that a framework hands a fixed set of buffers, real-time loops that
+ * must stay off the allocator.  dynamo_moe_forward takes its scratch from a workspace the caller
+ * allocated; this call needs none: the scan kernel's scratch lives in a fixed array inside the
+ * library (about 385 KiB of device memory per GPU that loads the library, held until exit).
+ *   router_logits : dev fp32 [T, n_experts]                       (input)
+ *   topk_idx      : dev int32 [T, top_k]   topk_w : dev fp32 [T, top_k]
+ *   expert_offsets: dev int32 [n_experts + 1]   perm : dev int32 [T * top_k]   (outputs, caller-owned)
+ * Same results as the routing outputs of dynamo_moe_forward.  Limits: T * top_k <=
+ * DYNAMO_NOALLOC_MAX_PAIRS (ERR_TOKENS beyond), n_experts <= 256, top_k <= 8 (ERR_SHAPE).
+ * Calls neither cudaMalloc nor cudaFree nor any allocating routine.  The first call on a device
+ * looks up the array's device address (with that device current); make that first call before
+ * starting any stream capture.  All calls share the one array, which keeps the previous call's
+ * contents (nothing needs clearing: every word read is written first); two calls that overlap on
+ * the GPU - different streams, or different threads - race on it, so order them on one stream.
+ * T = 0 is a no-op.  Asynchronous and stream-ordered like the other calls. */
+#define DYNAMO_NOALLOC_MAX_PAIRS 32768
+dynamo_status dynamo_route_permute_static(const float* router_logits, int32_t T, int32_t n_experts, int32_t top_k,
+                                          int32_t renormalize, int32_t* topk_idx, float* topk_w,
+                                          int32_t* expert_offsets, int32_t* perm, void* stream);
+
 #ifdef __cplusplus
 }
 #endif
