@@ -21,7 +21,7 @@ cudaError_t launch_scan(const WsDev& ws, int E, int Es, int k, cudaStream_t st);
 cudaError_t launch_gather(const LayerDev* L, const WsDev& ws, const void* x, cudaStream_t st);
 cudaError_t launch_combine(const WsDev& ws, int d, int k, int Es, void* y, int y_f32, long long split_stride,
                            cudaStream_t st);
-cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, int nt8, int n_tc, int n_rb, int ksplit,
+cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, int n_tc, int n_rb, int ksplit,
                               int n_experts, long long split_stride, int smem_bytes, cudaStream_t st);
 cudaError_t launch_switch(const SwitchLayers& layers, int n_layers, int E, const int32_t* staging, int per_layer_ints,
                           cudaStream_t st);
@@ -473,11 +473,10 @@ dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* ro
     CUDA_TRY(launch_route(router_logits, T, D.n_experts, D.top_k, D.renormalize, ws.topk_idx, ws.topk_w, st));
     CUDA_TRY(launch_scan(ws, D.n_experts, D.n_shared, D.top_k, st));
     CUDA_TRY(launch_gather(L, ws, x, st));
-    const int nt8 = T <= 8 ? 1 : (T <= 16 ? 2 : 4);
-    const int n_tc = (T + nt8 * 8 - 1) / (nt8 * 8);
+    const int n_tc = (T + 31) / 32;  // an expert holds at most T rows; chunks of 32 tokens
     const long long split_stride = (long long)ws.R * D.d_model;  // partials of one K split: [R][d]
-    CUDA_TRY(launch_ffn_stream(L, ws, 1, nt8, n_tc, ctx->host_layer.n_rb13, 1, n, split_stride, FFN_SMEM_BYTES, st));
-    CUDA_TRY(launch_ffn_stream(L, ws, 0, nt8, n_tc, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, FFN_SMEM_BYTES,
+    CUDA_TRY(launch_ffn_stream(L, ws, 1, n_tc, ctx->host_layer.n_rb13, 1, n, split_stride, FFN_SMEM_BYTES, st));
+    CUDA_TRY(launch_ffn_stream(L, ws, 0, n_tc, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, FFN_SMEM_BYTES,
                                st));
     CUDA_TRY(launch_combine(ws, D.d_model, D.top_k, D.n_shared, y, y_dtype == DYNAMO_F32, split_stride, st));
     ctx->launches += 6;

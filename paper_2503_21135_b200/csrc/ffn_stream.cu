@@ -1,24 +1,28 @@
 // Streaming grouped dequant-GEMM for small token counts per expert (decode path, and the generic
 // fallback for any size): HBM-bound, judged on packed-weight bytes per second.
 //
-// One CTA = one (expert, 256-row weight block, token chunk, K split).  A producer warp streams the
-// packed blocks (codes + params, contiguous per 256 x 128 block) and the matching activation slices
-// into a shared-memory ring with bulk async copies completing on mbarriers; eight consumer warps,
-// each owning two 16-row atoms, expand codes to fp16 integers with one LOP3/PRMT per pair
-// ((w >> sh) & mask | 0x6400.. = 1024 + code), issue mma.sync m16n8k16 (weights = A, tokens = B,
-// fp32 accumulate) and apply scale / zero once per group after the dot product:
-//     sum_k (s*q_k + m) x_k = s * sum_k (1024 + q_k) x_k + (m - 1024 s) * sum_k x_k .
+// One CTA = one (expert, 256-row weight block, chunk of <= 32 tokens, K split).  A producer warp
+// streams the packed blocks (codes + params, contiguous per 256 x 128 block) and the matching
+// activation slices into a shared-memory ring with bulk async copies completing on mbarriers; eight
+// consumer warps, each owning two 16-row atoms, turn codes into fp16 operands with ONE logic op per
+// register pair: a code field masked in place at bit offset o is the fp16 subnormal q * 2^(o-24),
+// and the activation slice already carries the factor 2^(bias-o) (see layout.cuh).  They issue
+// mma.sync m16n8k16 (weights = A, tokens = B, fp32 accumulate) and apply scale / zero once per
+// group after the dot product:
+//     sum_k (s*q_k + m) x_k = (s * 2^(24-bias)) * acc + m * sum_k x_k .
 // The per-group sums of x come precomputed with the activation slice.  Codes and activations are
 // exact in fp16, so the only roundings are the fp32 accumulation and the fp16 rounding of h.
+// The number of 8-token tiles (1..4) is chosen per CTA from the expert's actual token count.
 //
 // Gate/up variant: after the K loop the significant-channel correction runs as extra ring stages
 // (16 channels each): the fp16 tiles of the active cached channels are fetched through the slot ->
 // pool-position table and multiplied with the gathered activation columns into the same
-// accumulators; then SwiGLU, fp16 rounding of h, per-64 sums of h, coalesced store.
-// Down variant: writes fp32 partial outputs per K split.
+// accumulators; then SwiGLU, fp16 rounding of h, per-64 sums of h, coalesced store of h (scaled
+// for the down matrix).  Down variant: writes fp32 partial outputs per K split.
 #include <type_traits>
 
 #include "common.cuh"
+#include "layout.cuh"
 
 namespace dyn {
 
@@ -28,24 +32,34 @@ constexpr int SIG_TILE_STRIDE = 528;  // 512 B tile + 16 B pad: conflict-free ld
 constexpr int SIG_X_STRIDE = 48;      // 32 B of gathered activations per token + pad
 constexpr int SMEM_HEADER = 256;
 constexpr int MAX_STAGES = 8;
+constexpr int CHUNK_TOKENS = 32;
 
 __host__ __device__ inline int stage_bytes_for(int bits, int G, int NT) {
     const int b = block_bytes(bits, G) + NT * XROW;
     return (b + 127) & ~127;
 }
 
+// Packed codes of one atom for one half chunk (64 k = 4 MMA steps), per lane, plus the shifted copies.
 template <int BITS>
-struct Codes {
-    // packed codes of one atom for one half chunk (64 k = 4 MMA steps), per lane
-    static constexpr int NW = (BITS == 8) ? 8 : (BITS == 4 ? 4 : (BITS == 3 ? 3 : 2));
-    uint32_t w[NW];
-};
+struct Codes;
+template <>
+struct Codes<2> { uint32_t w[2], ws[2]; };
+template <>
+struct Codes<3> { uint32_t w[2], ws[2], t0[2], t1[2]; };
+template <>
+struct Codes<4> { uint32_t w[4], ws[4]; };
+template <>
+struct Codes<8> { uint32_t w[8]; };
+
+__device__ __forceinline__ uint32_t rotr32(uint32_t v, int n) { return __funnelshift_r(v, v, n); }
 
 template <int BITS>
 __device__ __forceinline__ void load_codes(Codes<BITS>& c, const uint8_t* atom, int lane, int half) {
     if constexpr (BITS == 4) {
         const uint4 v = *reinterpret_cast<const uint4*>(atom + half * 512 + lane * 16);
         c.w[0] = v.x; c.w[1] = v.y; c.w[2] = v.z; c.w[3] = v.w;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) c.ws[i] = c.w[i] >> 8;
     } else if constexpr (BITS == 8) {
         const uint4 v0 = *reinterpret_cast<const uint4*>(atom + (2 * half) * 512 + lane * 16);
         const uint4 v1 = *reinterpret_cast<const uint4*>(atom + (2 * half + 1) * 512 + lane * 16);
@@ -54,50 +68,63 @@ __device__ __forceinline__ void load_codes(Codes<BITS>& c, const uint8_t* atom, 
     } else if constexpr (BITS == 2) {
         const uint2 v = *reinterpret_cast<const uint2*>(atom + lane * 16 + half * 8);
         c.w[0] = v.x; c.w[1] = v.y;
+        c.ws[0] = v.x >> 10; c.ws[1] = v.y >> 10;
     } else {
         const uint2 v = *reinterpret_cast<const uint2*>(atom + lane * 16 + half * 8);
+        const uint2 hb = *reinterpret_cast<const uint2*>(atom + 512 + lane * 8);
         c.w[0] = v.x; c.w[1] = v.y;
-        c.w[2] = *reinterpret_cast<const uint32_t*>(atom + 512 + lane * 8 + half * 4);
+        c.ws[0] = v.x >> 8; c.ws[1] = v.y >> 8;
+        c.t0[0] = rotr32(hb.x, half * 8); c.t0[1] = rotr32(hb.y, half * 8);
+        c.t1[0] = rotr32(hb.x, half * 8 + 1); c.t1[1] = rotr32(hb.y, half * 8 + 1);
     }
 }
 
-__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t mask, uint32_t orv) {
-    uint32_t r;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(mask), "r"(orv));  // (a & b) | c
-    return r;
-}
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
     uint32_t r;
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
     return r;
 }
 
-// A-fragment registers (fp16 pairs 1024 + code) of step S4 (0..3) of the loaded half chunk.
+// A-fragment registers of step S4 (0..3) of the loaded half chunk: fp16 pairs q * 2^(o-24).
 template <int BITS, int S4>
 __device__ __forceinline__ void expand(const Codes<BITS>& c, uint32_t (&a)[4]) {
-    constexpr uint32_t MAGIC = 0x64006400u;
     if constexpr (BITS == 4) {
-        const uint32_t w = c.w[S4];
+        constexpr int jj = S4 >> 1;
 #pragma unroll
-        for (int ri = 0; ri < 4; ++ri) a[ri] = lop3_and_or(w >> (4 * ri), 0x000F000Fu, MAGIC);
+        for (int h = 0; h < 2; ++h) {
+            const int phi = 2 * (S4 & 1) + h;
+#pragma unroll
+            for (int rh = 0; rh < 2; ++rh) {
+                const uint32_t src = (phi < 2) ? c.w[rh * 2 + jj] : c.ws[rh * 2 + jj];
+                a[rh + 2 * h] = src & (0x000F000Fu << (4 * (phi & 1)));
+            }
+        }
     } else if constexpr (BITS == 8) {
         const uint32_t w0 = c.w[(S4 >> 1) * 4 + 2 * (S4 & 1)], w1 = c.w[(S4 >> 1) * 4 + 2 * (S4 & 1) + 1];
-        a[0] = prmt(w0, 0x64646464u, 0x4140u);
-        a[1] = prmt(w0, 0x64646464u, 0x4342u);
-        a[2] = prmt(w1, 0x64646464u, 0x4140u);
-        a[3] = prmt(w1, 0x64646464u, 0x4342u);
+        a[0] = prmt(w0, 0u, 0x4140u);
+        a[1] = prmt(w0, 0u, 0x4342u);
+        a[2] = prmt(w1, 0u, 0x4140u);
+        a[3] = prmt(w1, 0u, 0x4342u);
     } else if constexpr (BITS == 2) {
-        const uint32_t w = c.w[S4 >> 1];
 #pragma unroll
-        for (int ri = 0; ri < 4; ++ri) a[ri] = lop3_and_or(w >> (2 * ((S4 & 1) * 4 + ri)), 0x00030003u, MAGIC);
+        for (int h = 0; h < 2; ++h) {
+            const int phi = 2 * S4 + h;
+#pragma unroll
+            for (int rh = 0; rh < 2; ++rh)
+                a[rh + 2 * h] = (phi <= 4) ? (c.w[rh] & (0x00030003u << (2 * phi)))
+                                           : (c.ws[rh] & (0x00030003u << ((2 * phi - 10) & 31)));
+        }
     } else {
-        const uint32_t w = c.w[S4 >> 1], hb = c.w[2];
 #pragma unroll
-        for (int ri = 0; ri < 4; ++ri) {
-            const int R = ((S4 >> 1) & 1) * 8 + (S4 & 1) * 4 + ri;  // bit R -> position 2, bit R+16 -> position 18
-            const uint32_t t = (R >= 2) ? (hb >> ((R - 2) & 31)) : (hb << ((2 - R) & 31));
-            const uint32_t hi = lop3_and_or(t, 0x00040004u, MAGIC);
-            a[ri] = lop3_and_or(w >> (2 * ((S4 & 1) * 4 + ri)), 0x00030003u, hi);
+        for (int h = 0; h < 2; ++h) {
+            const int phi = 2 * S4 + h;
+            const int i = phi & 3;
+#pragma unroll
+            for (int rh = 0; rh < 2; ++rh) {
+                const uint32_t lo = (phi < 4) ? c.w[rh] : c.ws[rh];
+                const uint32_t hi = (phi < 4) ? c.t0[rh] : c.t1[rh];
+                a[rh + 2 * h] = (lo & (0x00030003u << (2 * i))) | (hi & (0x00040004u << (2 * i)));
+            }
         }
     }
 }
@@ -215,6 +242,9 @@ __device__ __forceinline__ void ffn_body(const FfnParams& p, const ExpertDev& ex
 #pragma unroll
             for (int c = 0; c < 4; ++c) total[a][j][c] = 0.f;
 
+    // exact power of two that undoes the operand scaling: codes enter as q*2^(o-24), activations as x*2^(bias-o)
+    const float unscale = __uint_as_float((uint32_t)(127 + 24 - x_scale_bias(BITS)) << 23);
+
     int it = 0;
     bool ok = true;
     for (int kc = kc0; kc < kc1; ++kc, ++it) {
@@ -271,8 +301,8 @@ __device__ __forceinline__ void ffn_body(const FfnParams& p, const ExpertDev& ex
                     const uint32_t p0 = prm[r0 * ngrp + g], p1 = prm[(r0 + 8) * ngrp + g];
                     const __half2 h0 = *reinterpret_cast<const __half2*>(&p0);
                     const __half2 h1 = *reinterpret_cast<const __half2*>(&p1);
-                    const float s0 = __low2float(h0), s1 = __low2float(h1);
-                    const float z0 = fmaf(-1024.f, s0, __high2float(h0)), z1 = fmaf(-1024.f, s1, __high2float(h1));
+                    const float s0 = __low2float(h0) * unscale, s1 = __low2float(h1) * unscale;
+                    const float m0 = __high2float(h0), m1 = __high2float(h1);
 #pragma unroll
                     for (int j = 0; j < NT8; ++j) {
                         const float* sp0 =
@@ -282,10 +312,10 @@ __device__ __forceinline__ void ffn_body(const FfnParams& p, const ExpertDev& ex
                         float xs0, xs1;
                         if (G == 64) { xs0 = sp0[half]; xs1 = sp1[half]; }
                         else { xs0 = sp0[0] + sp0[1]; xs1 = sp1[0] + sp1[1]; }
-                        total[a][j][0] += fmaf(s0, accg[a][j][0], z0 * xs0);
-                        total[a][j][1] += fmaf(s0, accg[a][j][1], z0 * xs1);
-                        total[a][j][2] += fmaf(s1, accg[a][j][2], z1 * xs0);
-                        total[a][j][3] += fmaf(s1, accg[a][j][3], z1 * xs1);
+                        total[a][j][0] += fmaf(s0, accg[a][j][0], m0 * xs0);
+                        total[a][j][1] += fmaf(s0, accg[a][j][1], m0 * xs1);
+                        total[a][j][2] += fmaf(s1, accg[a][j][2], m1 * xs0);
+                        total[a][j][3] += fmaf(s1, accg[a][j][3], m1 * xs1);
 #pragma unroll
                         for (int c = 0; c < 4; ++c) accg[a][j][c] = 0.f;
                     }
@@ -348,14 +378,22 @@ __device__ __forceinline__ void ffn_body(const FfnParams& p, const ExpertDev& ex
         if (lane == 0) mbar_arrive(done);
         if (!mbar_wait_bounded(done, 0, poison, p.ws.status) || *poison) return;
         const int n_rb = L->n_rb13;  // = chunks of the hidden axis
+        // this lane's four hidden indices 4*lane + {0..3}: the down matrix wants them scaled by 2^(bias-o)
+        const float sc0 = __uint_as_float((uint32_t)(127 + x_scale_exp(BITS, 4 * lane)) << 23);
+        const float sc1 = __uint_as_float((uint32_t)(127 + x_scale_exp(BITS, 4 * lane + 2)) << 23);
         for (int tok = warp; tok < nvalid; tok += CONSUMER_WARPS) {
             const uint2 v = *reinterpret_cast<const uint2*>(htile + tok * XROW + lane * 8);
             const __half2 a2 = *reinterpret_cast<const __half2*>(&v.x), b2 = *reinterpret_cast<const __half2*>(&v.y);
-            float sum = __low2float(a2) + __high2float(a2) + __low2float(b2) + __high2float(b2);
+            const float f0 = __low2float(a2), f1 = __high2float(a2), f2 = __low2float(b2), f3 = __high2float(b2);
+            float sum = f0 + f1 + f2 + f3;
 #pragma unroll
             for (int o = 8; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            const __half2 oa = __floats2half2_rn(f0 * sc0, f1 * sc0), ob = __floats2half2_rn(f2 * sc1, f3 * sc1);
+            uint2 ov;
+            ov.x = *reinterpret_cast<const uint32_t*>(&oa);
+            ov.y = *reinterpret_cast<const uint32_t*>(&ob);
             uint8_t* dst = p.ws.hbuf + ((size_t)(row0 + tok) * n_rb + rb) * XROW;
-            *reinterpret_cast<uint2*>(dst + lane * 8) = v;
+            *reinterpret_cast<uint2*>(dst + lane * 8) = ov;
             if ((lane & 15) == 0) *reinterpret_cast<float*>(dst + XROW_SUM_OFF + (lane >> 4) * 4) = sum;
         }
     } else {
@@ -374,39 +412,48 @@ __device__ __forceinline__ void ffn_body(const FfnParams& p, const ExpertDev& ex
     }
 }
 
-template <int NT8, bool GATEUP>
+template <int BITS, bool GATEUP>
+__device__ __forceinline__ void ffn_dispatch_tiles(const FfnParams& p, const ExpertDev& ex, int e, int rb, int split,
+                                                   int row0, int nvalid, uint8_t* smem) {
+    const int nt8 = (nvalid + 7) >> 3;
+    if (nt8 == 1) ffn_body<BITS, 1, GATEUP>(p, ex, e, rb, split, row0, nvalid, smem);
+    else if (nt8 == 2) ffn_body<BITS, 2, GATEUP>(p, ex, e, rb, split, row0, nvalid, smem);
+    else if (nt8 == 3) ffn_body<BITS, 3, GATEUP>(p, ex, e, rb, split, row0, nvalid, smem);
+    else ffn_body<BITS, 4, GATEUP>(p, ex, e, rb, split, row0, nvalid, smem);
+}
+
+template <bool GATEUP>
 __global__ void __launch_bounds__(FFN_THREADS, 2) ffn_stream_kernel(const FfnParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
-    constexpr int NT = NT8 * 8;
     const LayerDev* L = p.L;
     const int e = L->order[blockIdx.y];
     const int tc = blockIdx.x % p.n_tc;
     const int rbs = blockIdx.x / p.n_tc;
     const int rb = rbs / p.ksplit, split = rbs % p.ksplit;
     const int off0 = p.ws.offsets[e], off1 = p.ws.offsets[e + 1];
-    const int row0 = off0 + tc * NT;
+    const int row0 = off0 + tc * CHUNK_TOKENS;
     if (row0 >= off1) return;
-    const int nvalid = min(NT, off1 - row0);
+    const int nvalid = min(CHUNK_TOKENS, off1 - row0);
     const ExpertDev& ex = L->ex[e];
     switch (ex.bits) {
-        case 2: ffn_body<2, NT8, GATEUP>(p, ex, e, rb, split, row0, nvalid, smem); break;
-        case 3: ffn_body<3, NT8, GATEUP>(p, ex, e, rb, split, row0, nvalid, smem); break;
-        case 4: ffn_body<4, NT8, GATEUP>(p, ex, e, rb, split, row0, nvalid, smem); break;
-        default: ffn_body<8, NT8, GATEUP>(p, ex, e, rb, split, row0, nvalid, smem); break;
+        case 2: ffn_dispatch_tiles<2, GATEUP>(p, ex, e, rb, split, row0, nvalid, smem); break;
+        case 3: ffn_dispatch_tiles<3, GATEUP>(p, ex, e, rb, split, row0, nvalid, smem); break;
+        case 4: ffn_dispatch_tiles<4, GATEUP>(p, ex, e, rb, split, row0, nvalid, smem); break;
+        default: ffn_dispatch_tiles<8, GATEUP>(p, ex, e, rb, split, row0, nvalid, smem); break;
     }
 }
 
-template <int NT8, bool GATEUP>
+template <bool GATEUP>
 static cudaError_t launch_one(const FfnParams& p, dim3 grid, cudaStream_t st) {
-    cudaError_t err = cudaFuncSetAttribute(ffn_stream_kernel<NT8, GATEUP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t err = cudaFuncSetAttribute(ffn_stream_kernel<GATEUP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            p.smem_bytes);
     if (err != cudaSuccess) return err;
-    ffn_stream_kernel<NT8, GATEUP><<<grid, FFN_THREADS, p.smem_bytes, st>>>(p);
+    ffn_stream_kernel<GATEUP><<<grid, FFN_THREADS, p.smem_bytes, st>>>(p);
     return cudaGetLastError();
 }
 
-// nt8: token tiles of 8 per chunk (1, 2 or 4).  n_rb: weight row blocks; n_experts: experts in L->order.
-cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, int nt8, int n_tc, int n_rb, int ksplit,
+// n_tc: 32-token chunks per expert launched; n_rb: weight row blocks; n_experts: experts in L->order.
+cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, int n_tc, int n_rb, int ksplit,
                               int n_experts, long long split_stride, int smem_bytes, cudaStream_t st) {
     FfnParams p;
     p.L = L;
@@ -416,14 +463,7 @@ cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, in
     p.split_stride = split_stride;
     p.smem_bytes = smem_bytes;
     dim3 grid((unsigned)(n_tc * n_rb * ksplit), (unsigned)n_experts);
-    if (gateup) {
-        if (nt8 == 1) return launch_one<1, true>(p, grid, st);
-        if (nt8 == 2) return launch_one<2, true>(p, grid, st);
-        return launch_one<4, true>(p, grid, st);
-    }
-    if (nt8 == 1) return launch_one<1, false>(p, grid, st);
-    if (nt8 == 2) return launch_one<2, false>(p, grid, st);
-    return launch_one<4, false>(p, grid, st);
+    return gateup ? launch_one<true>(p, grid, st) : launch_one<false>(p, grid, st);
 }
 
 }  // namespace dyn

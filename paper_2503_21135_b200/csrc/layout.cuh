@@ -1,20 +1,30 @@
-// Where a logical code lives inside a packed atom (16 rows x 128 k of one bit-width).
+// Where a logical code lives inside a packed atom (16 rows x 128 k of one bit-width), and the
+// power-of-two scale the activations carry so that codes can be used where they lie.
 //
 // The layout is "fragment native" for mma.sync m16n8k16 with the weights as the A operand: lane
 // (gid = lane/4, tid4 = lane%4) of a warp owns rows gid and gid+8 of the atom and, in MMA step
-// s (k in [16s, 16s+16)), the four consecutive k = 16s + 4*tid4 + {0,1,2,3}.  Its 64 codes are
-// contiguous per lane so that one or two 16-byte shared-memory loads fetch them, and the fields
-// of a 32-bit word are ordered so that ((w >> shift) & mask) | 0x64006400 is directly the fp16
-// pair (1024 + code_even, 1024 + code_odd) of one A-fragment register:
+// s (k in [16s, 16s+16)), the four consecutive k = 16s + 4*tid4 + {0,1,2,3}.  A-fragment register
+// ri = rowhalf + 2*h holds (row gid + 8*rowhalf, k = 16s + 4*tid4 + 2*h + {0,1}) as an fp16 pair.
 //
-//   A register ri = rowhalf + 2*h  holds (row gid + 8*rowhalf, k = 16s + 4*tid4 + 2*h + {0,1}).
+// A code is NOT shifted down to bit 0 before use.  A field of width b at bit offset o (o + b <= 10)
+// of a 16-bit half, masked in place, is the fp16 SUBNORMAL q * 2^(o-24); the matching activation is
+// stored pre-multiplied by 2^(bias - o), so the product is q * x * 2^(bias-24) whatever o is, and one
+// AND per register pair (plus one shift per 32-bit word to bring the upper fields below bit 10)
+// replaces shift + mask + or.  The offset o of a k must not depend on the row (the B fragment is
+// shared by all rows), so the two row halves live in different words:
 //
-//   4-bit: atom = 2 planes x [32 lanes x 16 B]; plane s/4, word s%4; nibble ri (even k) and
-//          nibble ri+4 (odd k).
-//   2-bit: atom = [32 lanes x 16 B]; word s/2; 2-bit field (s%2)*4 + ri (even k), +8 (odd k).
-//   8-bit: atom = 4 planes x [32 lanes x 16 B]; plane s/2, word 2*(s%2) + h; byte 2*rowhalf + odd.
-//   3-bit: the low two bits exactly as a 2-bit atom (512 B), followed by a 1-bit plane
-//          [32 lanes x 8 B]: word s/4, bit R (even k) and R+16 (odd k), R = ((s/2)%2)*8 + (s%2)*4 + ri.
+//   2-bit: atom = [32 lanes x 16 B]; word jh*2 + rowhalf (jh = s/4, the 64-k half chunk);
+//          field phi = 2*(s%4) + h at bits [2phi, 2phi+2) (even k) and +16 (odd k);
+//          phi <= 4 used in place (o = 2phi), phi >= 5 after >> 10 (o = 2phi - 10).
+//   3-bit: low two bits stored exactly as a 2-bit atom but used as phi <= 3 in place (o = 2phi),
+//          phi >= 4 after >> 8 (o = 2phi - 8); then a 1-bit plane [32 lanes x 8 B], word = rowhalf:
+//          the high bit of field (jh, phi) must land on bit o+2 (even k) / o+18 (odd k) after a
+//          rotation by rot = {0, 1, 8, 9}[2*jh + phi/4], i.e. it is stored at bit (o + 2 + 16*odd + rot) % 32.
+//   4-bit: atom = 2 planes (= half chunks) x [32 lanes x 16 B]; word rowhalf*2 + (s%4)/2;
+//          nibble phi = 2*(s%2) + h at bits [4phi, 4phi+4) (even k) and +16 (odd k);
+//          phi <= 1 in place (o = 4phi), phi >= 2 after >> 8 (o = 4phi - 8): o = 4h.
+//   8-bit: atom = 4 planes x [32 lanes x 16 B]; plane s/2, word 2*(s%2) + h; byte 2*rowhalf + odd
+//          (expanded with one byte permute per pair; o = 0).
 #pragma once
 #include <stdint.h>
 
@@ -32,26 +42,45 @@ __host__ __device__ inline CodeLoc code_loc(int bits, int r, int kk, int part) {
     const int s = kk >> 4, kq = kk & 15;
     const int tid4 = kq >> 2, h = (kq >> 1) & 1, odd = kq & 1;
     const int lane = gid * 4 + tid4;
-    const int ri = rowhalf + 2 * h;
+    const int jh = s >> 2, s4 = s & 3;
     CodeLoc L;
     if (bits == 4) {
-        L.byte_off = (s >> 2) * 512 + lane * 16 + (s & 3) * 4;
-        L.shift = 4 * (ri + 4 * odd);
+        const int phi = 2 * (s4 & 1) + h;
+        L.byte_off = jh * 512 + lane * 16 + (rowhalf * 2 + (s4 >> 1)) * 4;
+        L.shift = 4 * phi + 16 * odd;
         L.width = 4;
     } else if (bits == 8) {
         L.byte_off = (s >> 1) * 512 + lane * 16 + (2 * (s & 1) + h) * 4;
         L.shift = 8 * (2 * rowhalf + odd);
         L.width = 8;
     } else if (bits == 2 || (bits == 3 && part == 0)) {
-        L.byte_off = lane * 16 + (s >> 1) * 4;
-        L.shift = 2 * ((s & 1) * 4 + ri + 8 * odd);
+        const int phi = 2 * s4 + h;
+        L.byte_off = lane * 16 + (jh * 2 + rowhalf) * 4;
+        L.shift = 2 * phi + 16 * odd;
         L.width = 2;
     } else {  // 3-bit, high bit plane
-        L.byte_off = 512 + lane * 8 + (s >> 2) * 4;
-        L.shift = ((s >> 1) & 1) * 8 + (s & 1) * 4 + ri + 16 * odd;
+        const int phi = 2 * s4 + h;
+        const int o = 2 * (phi & 3);
+        const int st = 2 * jh + (phi >> 2);
+        const int rot = (st & 1) + 8 * (st >> 1);
+        L.byte_off = 512 + lane * 8 + rowhalf * 4;
+        L.shift = (o + 2 + 16 * odd + rot) & 31;
         L.width = 1;
     }
     return L;
+}
+
+// Activations feeding a matrix packed at `bits` are stored multiplied by 2^x_scale_exp(bits, k):
+// bias - o(k), with o the in-place bit offset of the code of input index k (periodic in k mod 64).
+__host__ __device__ inline int x_scale_bias(int bits) { return bits == 2 ? 4 : (bits == 3 ? 3 : (bits == 4 ? 2 : 0)); }
+__host__ __device__ inline int x_scale_exp(int bits, int k) {
+    const int s4 = (k >> 4) & 3, h = (k >> 1) & 1;
+    const int phi = 2 * s4 + h;
+    int o = 0;
+    if (bits == 2) o = phi <= 4 ? 2 * phi : 2 * phi - 10;
+    else if (bits == 3) o = 2 * (phi & 3);
+    else if (bits == 4) o = 4 * h;
+    return x_scale_bias(bits) - o;
 }
 
 }  // namespace dyn

@@ -7,6 +7,7 @@
 //           experts (they are served by the 8-bit path), per-64 sums, plus the gathered significant columns.
 // combine : y[t] = sum_j w[t,j] * Y[pos(t,j)] + sum_shared Y[pos], fp32, fixed order.
 #include "common.cuh"
+#include "layout.cuh"
 
 namespace dyn {
 
@@ -123,18 +124,22 @@ __global__ void __launch_bounds__(1024) scan_kernel(WsDev ws, int E, int Es, int
     }
 }
 
-// One warp per sorted row.
+// One CTA per sorted row; warp w converts chunks w, w+8, ...  The fp16 activations are stored
+// multiplied by 2^x_scale_exp(bits of the row's expert, k) so that the FFN kernel can use packed codes
+// in place; the per-64 sums are of the unscaled fp16 values.
 __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict__ L, WsDev ws,
                                                      const __nv_bfloat16* __restrict__ x) {
-    const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-    if (row >= ws.R) return;
+    const int row = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t = ws.row_token[row], e = ws.row_expert[row];
     const int d = L->d;
+    const int bits = L->ex[e].bits;
     const bool sw = L->ex[e].switchable != 0;
     const uint32_t* mask = sw ? (L->sigmask + (long long)e * (d / 32)) : nullptr;
     const __nv_bfloat16* xr = x + (long long)t * d;
     uint8_t* out = ws.xperm + (long long)row * (d / KC) * XROW;
-    for (int c = 0; c < d / KC; ++c) {
+    const float sc0 = __uint_as_float((uint32_t)(127 + x_scale_exp(bits, 4 * lane)) << 23);
+    const float sc1 = __uint_as_float((uint32_t)(127 + x_scale_exp(bits, 4 * lane + 2)) << 23);
+    for (int c = warp; c < d / KC; c += 8) {
         const int k0 = c * KC + lane * 4;
         const uint2 raw = *reinterpret_cast<const uint2*>(xr + k0);
         const __nv_bfloat162 p0 = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
@@ -146,60 +151,61 @@ __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict_
             for (int i = 0; i < 4; ++i)
                 if ((mw >> i) & 1u) v[i] = 0.f;
         }
-        __half h[4];
+        float hv[4];
         float sum = 0.f;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            h[i] = __float2half_rn(v[i]);
-            sum += __half2float(h[i]);
+            hv[i] = __half2float(__float2half_rn(v[i]));
+            sum += hv[i];
         }
         // sum over the 16 lanes of each half chunk (64 k), fixed butterfly order
 #pragma unroll
         for (int o = 8; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        const __half2 oa = __floats2half2_rn(hv[0] * sc0, hv[1] * sc0), ob = __floats2half2_rn(hv[2] * sc1, hv[3] * sc1);
         uint2 packed;
-        packed.x = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
-        packed.y = (uint32_t)__half_as_ushort(h[2]) | ((uint32_t)__half_as_ushort(h[3]) << 16);
+        packed.x = *reinterpret_cast<const uint32_t*>(&oa);
+        packed.y = *reinterpret_cast<const uint32_t*>(&ob);
         *reinterpret_cast<uint2*>(out + (long long)c * XROW + lane * 8) = packed;
         if ((lane & 15) == 0)
             *reinterpret_cast<float*>(out + (long long)c * XROW + XROW_SUM_OFF + (lane >> 4) * 4) = sum;
     }
-    // gathered significant columns
+    // gathered significant columns (unscaled)
     const int S_pad = L->S_pad;
     const int cnt = sw ? L->sig_cnt[e] : 0;
-    for (int j = lane; j < S_pad; j += 32) {
+    for (int j = threadIdx.x; j < S_pad; j += blockDim.x) {
         __half hv = __float2half_rn(0.f);
         if (j < cnt) hv = __float2half_rn(__bfloat162float(xr[L->sig_chan[e * S_pad + j]]));
         ws.xsig[(long long)row * S_pad + j] = hv;
     }
 }
 
-// One CTA per token.
+// grid (T, ceil(d / 1024)): each thread owns four output columns of one token.
 __global__ void __launch_bounds__(256) combine_kernel(WsDev ws, int d, int k, int Es, void* __restrict__ y,
                                                       int y_f32, long long split_stride) {
     const int t = blockIdx.x;
     const int kk = k + Es;
-    for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int j = 0; j < kk; ++j) {
-            const int r = ws.pos[t * kk + j];
-            const float w = (j < k) ? ws.topk_w[t * k + j] : 1.0f;
-            float s[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int sp = 0; sp < ws.ksplit; ++sp) {
-                const float4 v = *reinterpret_cast<const float4*>(ws.ypart + sp * split_stride + (long long)r * d + c);
-                s[0] += v.x; s[1] += v.y; s[2] += v.z; s[3] += v.w;
-            }
+    const int c = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
+    if (c >= d) return;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int j = 0; j < kk; ++j) {
+        const int r = ws.pos[t * kk + j];
+        const float w = (j < k) ? ws.topk_w[t * k + j] : 1.0f;
+        float s[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int sp = 0; sp < ws.ksplit; ++sp) {
+            const float4 v = *reinterpret_cast<const float4*>(ws.ypart + sp * split_stride + (long long)r * d + c);
+            s[0] += v.x; s[1] += v.y; s[2] += v.z; s[3] += v.w;
+        }
 #pragma unroll
-            for (int i = 0; i < 4; ++i) acc[i] = fmaf(w, s[i], acc[i]);
-        }
-        if (y_f32) {
-            *reinterpret_cast<float4*>((float*)y + (long long)t * d + c) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-        } else {
-            __nv_bfloat162 a = __floats2bfloat162_rn(acc[0], acc[1]), b = __floats2bfloat162_rn(acc[2], acc[3]);
-            uint2 o;
-            o.x = *reinterpret_cast<uint32_t*>(&a);
-            o.y = *reinterpret_cast<uint32_t*>(&b);
-            *reinterpret_cast<uint2*>((__nv_bfloat16*)y + (long long)t * d + c) = o;
-        }
+        for (int i = 0; i < 4; ++i) acc[i] = fmaf(w, s[i], acc[i]);
+    }
+    if (y_f32) {
+        *reinterpret_cast<float4*>((float*)y + (long long)t * d + c) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    } else {
+        __nv_bfloat162 a = __floats2bfloat162_rn(acc[0], acc[1]), b = __floats2bfloat162_rn(acc[2], acc[3]);
+        uint2 o;
+        o.x = *reinterpret_cast<uint32_t*>(&a);
+        o.y = *reinterpret_cast<uint32_t*>(&b);
+        *reinterpret_cast<uint2*>((__nv_bfloat16*)y + (long long)t * d + c) = o;
     }
 }
 
@@ -214,12 +220,12 @@ cudaError_t launch_scan(const WsDev& ws, int E, int Es, int k, cudaStream_t st) 
     return cudaGetLastError();
 }
 cudaError_t launch_gather(const LayerDev* L, const WsDev& ws, const void* x, cudaStream_t st) {
-    gather_kernel<<<(ws.R + 7) / 8, 256, 0, st>>>(L, ws, (const __nv_bfloat16*)x);
+    gather_kernel<<<ws.R, 256, 0, st>>>(L, ws, (const __nv_bfloat16*)x);
     return cudaGetLastError();
 }
 cudaError_t launch_combine(const WsDev& ws, int d, int k, int Es, void* y, int y_f32, long long split_stride,
                            cudaStream_t st) {
-    combine_kernel<<<ws.T, 256, 0, st>>>(ws, d, k, Es, y, y_f32, split_stride);
+    combine_kernel<<<dim3((unsigned)ws.T, (unsigned)((d + 1023) / 1024)), 256, 0, st>>>(ws, d, k, Es, y, y_f32, split_stride);
     return cudaGetLastError();
 }
 
