@@ -171,6 +171,11 @@ dynamo_status dynamo_expert_stream_bytes(dynamo_ctx* ctx, int32_t expert, size_t
  * clears it. */
 dynamo_status dynamo_poll_status(dynamo_ctx* ctx, void* stream);
 
+/* Measurement hook: three cudaEvent_t handles (any may be NULL) that every following forward records on
+ * its stream before the gate/up FFN launch, after it, and after the down FFN launch, so that a
+ * harness can time the dominant kernels in place.  Pass NULLs to switch it off. */
+dynamo_status dynamo_set_profile_events(dynamo_ctx* ctx, void* before_gateup, void* after_gateup, void* after_down);
+
 /* Number of kernels the library launched through this context since creation (host counter). */
 int64_t dynamo_kernel_launches(const dynamo_ctx* ctx);
 

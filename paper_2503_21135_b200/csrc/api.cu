@@ -164,6 +164,7 @@ struct dynamo_ctx {
     LayerDev host_layer;                         // host mirror of the arena header
     int switch_mode = DYNAMO_SWITCH_SELECT;
     int64_t launches = 0;
+    cudaEvent_t prof_ev[3] = {nullptr, nullptr, nullptr};  // optional: before gate/up, after gate/up, after down
     std::vector<int32_t> upload;                 // scratch for switch uploads
 };
 
@@ -282,6 +283,14 @@ dynamo_status dynamo_arena_bytes(const dynamo_layer_desc* desc, const int32_t* b
 }
 
 int64_t dynamo_kernel_launches(const dynamo_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+dynamo_status dynamo_set_profile_events(dynamo_ctx* ctx, void* before_gateup, void* after_gateup, void* after_down) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    ctx->prof_ev[0] = (cudaEvent_t)before_gateup;
+    ctx->prof_ev[1] = (cudaEvent_t)after_gateup;
+    ctx->prof_ev[2] = (cudaEvent_t)after_down;
+    return DYNAMO_OK;
+}
 
 dynamo_status dynamo_set_switch_mode(dynamo_ctx* ctx, int32_t mode) {
     if (!ctx) return DYNAMO_ERR_NULL;
@@ -475,9 +484,12 @@ dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* ro
     CUDA_TRY(launch_gather(L, ws, x, st));
     const int n_tc = (T + 31) / 32;  // an expert holds at most T rows; chunks of 32 tokens
     const long long split_stride = (long long)ws.R * D.d_model;  // partials of one K split: [R][d]
+    if (ctx->prof_ev[0]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[0], st));
     CUDA_TRY(launch_ffn_stream(L, ws, 1, n_tc, ctx->host_layer.n_rb13, 1, n, split_stride, FFN_SMEM_BYTES, st));
+    if (ctx->prof_ev[1]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[1], st));
     CUDA_TRY(launch_ffn_stream(L, ws, 0, n_tc, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, FFN_SMEM_BYTES,
                                st));
+    if (ctx->prof_ev[2]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[2], st));
     CUDA_TRY(launch_combine(ws, D.d_model, D.top_k, D.n_shared, y, y_dtype == DYNAMO_F32, split_stride, st));
     ctx->launches += 6;
     if (dbg) {
