@@ -1,0 +1,114 @@
+"""GPU parity at the full sizes of the prefill (config 3), fine-grained (config 4) and switch-stress
+(config 5) workloads.  Routing, permutation and sampled codes are compared bit-exactly in full; the FFN
+output is compared on a seeded, expert-stratified token subset that the float64 oracle can compute in
+seconds (the subset rule: all experts touched, the two least-loaded experts over-sampled)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import make_gpu_layer, make_inputs, make_oracle_layer, rel_err, stratified_tokens
+from paper_2503_21135_b200 import binding
+from paper_2503_21135_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+
+
+def _check_forward(cfg, gpu, ora, T, n_sample, step=0, layer=0):
+    x, lg = wl.activations(cfg, T, layer, step), wl.router_logits(cfg, T, layer, step)
+    y, dbg = gpu.forward(x.cuda(), lg.cuda(), binding.F32, debug=True)
+    torch.cuda.synchronize()
+    assert gpu.poll_status() == 0
+    idx, w = oracle.route(lg.numpy(), cfg.top_k)
+    offsets, perm = oracle.permute(idx, cfg.n_experts)
+    assert np.array_equal(dbg["idx"].cpu().numpy(), idx)
+    assert np.array_equal(dbg["offsets"].cpu().numpy(), offsets)
+    assert np.array_equal(dbg["perm"].cpu().numpy(), perm)
+    assert np.max(np.abs(dbg["w"].cpu().numpy().astype(np.float64) - w)) <= 1e-6
+    toks = stratified_tokens(idx, cfg.n_experts, n_sample, seed=step) if n_sample < T else np.arange(T, dtype=np.int32)
+    ref = ora.forward(oracle.as_u16(x), lg.numpy(), tokens=toks)["y"][toks]
+    got = y.cpu().numpy()[toks]
+    assert np.all(np.isfinite(y.cpu().numpy()))
+    err = rel_err(got, ref)
+    print(f"{cfg.name} T={T} sample={len(toks)}: max|gpu-oracle|/rms = {err:.3e}")
+    assert err <= TOL, err
+    return idx
+
+
+def test_prefill_config():
+    cfg = wl.CONFIGS["prefill"]
+    wg, wu, wd, bits, pool, sets = make_inputs(cfg)
+    assert bits.tolist() == [3, 3, 3, 3, 4, 4, 4, 8]
+    gpu = make_gpu_layer(cfg, wg, wu, wd, bits, pool, max_tokens=4096)
+    ora = make_oracle_layer(cfg, wg, wu, wd, bits)
+    gpu.set_channel_switch(sets)
+    ora.set_channel_switch(sets)
+    # sampled codes: one expert per bit-width
+    for e in (0, 4, 7):
+        q, s, m = gpu.export_codes(e, binding.MAT_DOWN)
+        assert torch.equal(q.cpu(), torch.from_numpy(ora.base[e][2].q))
+        assert np.array_equal(s.cpu().numpy().view(np.uint16), ora.base[e][2].s)
+    idx = _check_forward(cfg, gpu, ora, 4096, 96)
+    counts = np.bincount(idx.ravel(), minlength=8)
+    assert counts[7] == counts.max() and counts[7] > 2 * counts[0]        # Zipf skew: expert 7 most loaded
+    # a ragged token count that leaves partial 32-token chunks in every expert
+    _check_forward(cfg, gpu, ora, 1000, 48, step=1)
+
+
+def test_finegrained_config_with_shared_experts():
+    cfg = wl.CONFIGS["finegrained"]
+    wg, wu, wd, bits, pool, sets = make_inputs(cfg)
+    assert sorted(bits[:64].tolist(), reverse=True) == [4] * 16 + [3] * 24 + [2] * 24 and bits[64:].tolist() == [8, 8]
+    gpu = make_gpu_layer(cfg, wg, wu, wd, bits, pool, max_tokens=2048)
+    ora = make_oracle_layer(cfg, wg, wu, wd, bits)
+    gpu.set_channel_switch(sets)
+    ora.set_channel_switch(sets)
+    for e in (0, 20, 50, 65):
+        for mat in (binding.MAT_GATE, binding.MAT_DOWN):
+            q, s, m = gpu.export_codes(e, mat)
+            assert torch.equal(q.cpu(), torch.from_numpy(ora.base[e][mat].q))
+            assert np.array_equal(m.cpu().numpy().view(np.uint16), ora.base[e][mat].m)
+    idx = _check_forward(cfg, gpu, ora, 2048, 80)
+    counts = np.bincount(idx.ravel(), minlength=64)
+    assert counts.min() <= 8 and counts.max() >= 1000                     # from decode-like to prefill-like experts
+    _check_forward(cfg, gpu, ora, 37, 37, step=2)
+
+
+def test_switch_stress_stack():
+    cfg = wl.CONFIGS["switch"]
+    n_layers, T = 3, 16
+    gpus, oras, pools, cur, ws = [], [], [], [], None
+    for l in range(n_layers):
+        wg, wu, wd, bits, pool, sets = make_inputs(cfg, layer=l)
+        g = make_gpu_layer(cfg, wg, wu, wd, bits, pool, max_tokens=T, workspace=ws)
+        ws = g.workspace
+        gpus.append(g)
+        oras.append(make_oracle_layer(cfg, wg, wu, wd, bits))
+        pools.append(pool)
+        cur.append(sets)
+    binding.set_channel_switch_many(gpus, cur)
+    for l in range(n_layers):
+        oras[l].set_channel_switch(cur[l])
+    step = 0
+    for event in range(3):
+        for l in range(n_layers):
+            _check_forward(cfg, gpus[l], oras[l], T, T, step=step, layer=l)
+        step += 8
+        new = [wl.switch_event(cfg, pools[l], cur[l], l, event) for l in range(n_layers)]
+        for l in range(n_layers):
+            for e in range(cfg.n_experts):
+                assert len(np.setdiff1d(new[l][e], cur[l][e])) == 16       # 25 % of 64 swapped
+        binding.set_channel_switch_many(gpus, new)                         # one upload + one launch for the stack
+        for l in range(n_layers):
+            oras[l].set_channel_switch(new[l])
+        cur = new
+    # all-or-nothing: one bad layer rejects the whole event and nothing changes
+    x, lg = wl.activations(cfg, T, 0, 99).cuda(), wl.router_logits(cfg, T, 0, 99).cuda()
+    y0 = gpus[0].forward(x, lg).clone()
+    bad = [list(s) for s in cur]
+    bad[n_layers - 1][3] = np.array([int(np.setdiff1d(np.arange(cfg.d_model), pools[n_layers - 1][3])[0])], np.int32)
+    with pytest.raises(binding.DynamoError) as ei:
+        binding.set_channel_switch_many(gpus, bad)
+    assert ei.value.status == 8
+    assert torch.equal(gpus[0].forward(x, lg), y0)
