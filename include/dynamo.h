@@ -171,6 +171,11 @@ dynamo_status dynamo_expert_stream_bytes(dynamo_ctx* ctx, int32_t expert, size_t
  * clears it. */
 dynamo_status dynamo_poll_status(dynamo_ctx* ctx, void* stream);
 
+/* Path selection: experts that receive more than `rows` tokens in a forward run on the tcgen05
+ * (tensor-memory) kernel, the others on the streaming kernel.  Default 32 (also the maximum);
+ * 0 switches the tcgen05 path off.  Both paths implement the same arithmetic definition. */
+dynamo_status dynamo_set_tc_min_rows(dynamo_ctx* ctx, int32_t rows);
+
 /* Measurement hook: three cudaEvent_t handles (any may be NULL) that every following forward records on
  * its stream before the gate/up FFN launch, after it, and after the down FFN launch, so that a
  * harness can time the dominant kernels in place.  Pass NULLs to switch it off. */
@@ -187,7 +192,7 @@ const char* dynamo_status_str(dynamo_status s);
  * is being captured, plugins that a framework hands a fixed set of buffers, real-time loops that
  * must stay off the allocator.  dynamo_moe_forward takes its scratch from a workspace the caller
  * allocated; this call needs none: the scan kernel's scratch lives in a fixed array inside the
- * library (about 385 KiB of device memory per GPU that loads the library, held until exit).
+ * library (about 400 KiB of device memory per GPU that loads the library, held until exit).
  *   router_logits : dev fp32 [T, n_experts]                       (input)
  *   topk_idx      : dev int32 [T, top_k]   topk_w : dev fp32 [T, top_k]
  *   expert_offsets: dev int32 [n_experts + 1]   perm : dev int32 [T * top_k]   (outputs, caller-owned)

@@ -31,7 +31,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_BITS", "ERR_ALIGN", "ERR_ARE
 EXPORTED = ["dynamo_create", "dynamo_destroy", "dynamo_arena_bytes", "dynamo_pack_experts",
             "dynamo_set_channel_switch", "dynamo_set_channel_switch_many", "dynamo_set_switch_mode",
             "dynamo_moe_forward", "dynamo_moe_forward_host", "dynamo_export_codes", "dynamo_expert_stream_bytes",
-            "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_route_permute_static", "dynamo_kernel_launches", "dynamo_status_str"]
+            "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_route_permute_static", "dynamo_kernel_launches", "dynamo_status_str"]
 
 
 class LayerDesc(ctypes.Structure):
@@ -74,6 +74,7 @@ def load():
         L.dynamo_expert_stream_bytes.argtypes = [vp, i32, ctypes.POINTER(sz)]
         L.dynamo_poll_status.argtypes = [vp, vp]
         L.dynamo_set_profile_events.argtypes = [vp, vp, vp, vp]
+        L.dynamo_set_tc_min_rows.argtypes = [vp, i32]
         L.dynamo_route_permute_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
         L.dynamo_kernel_launches.argtypes = [vp]
         L.dynamo_kernel_launches.restype = ctypes.c_int64
@@ -153,6 +154,10 @@ def dynamo_expert_stream_bytes(ctx, expert: int):
 
 def dynamo_poll_status(ctx, stream) -> int:
     return load().dynamo_poll_status(ctx, stream)
+
+
+def dynamo_set_tc_min_rows(ctx, rows: int) -> int:
+    return load().dynamo_set_tc_min_rows(ctx, rows)
 
 
 def dynamo_set_profile_events(ctx, e0, e1, e2) -> int:
@@ -288,6 +293,9 @@ class DynamoLayer:
         st, b = dynamo_expert_stream_bytes(self.ctx, expert)
         _check(st, "dynamo_expert_stream_bytes")
         return b
+
+    def set_tc_min_rows(self, rows: int):
+        _check(dynamo_set_tc_min_rows(self.ctx, rows), "dynamo_set_tc_min_rows")
 
     def set_profile_events(self, events=None):
         """events: three torch.cuda.Event (already recorded once, so that their handles exist) or None."""

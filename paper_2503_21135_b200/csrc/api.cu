@@ -23,6 +23,8 @@ cudaError_t launch_combine(const WsDev& ws, int d, int k, int Es, void* y, int y
                            cudaStream_t st);
 cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, int n_tc, int n_rb, int ksplit,
                               int n_experts, long long split_stride, int smem_bytes, cudaStream_t st);
+cudaError_t launch_ffn_tc(const LayerDev* L, const WsDev& ws, int gateup, int n_tt, int n_rb, int n_experts,
+                          cudaStream_t st);
 cudaError_t launch_switch(const SwitchLayers& layers, int n_layers, int E, const int32_t* staging, int per_layer_ints,
                           cudaStream_t st);
 }  // namespace dyn
@@ -48,7 +50,8 @@ struct ArenaLayout {
 };
 
 struct WsLayout {
-    size_t status, counts, offsets, topk_idx, topk_w, perm, pos, row_token, row_expert, xperm, xsig, hbuf, ypart,
+    size_t status, counts, offsets, off_pad, topk_idx, topk_w, perm, pos, row_token, row_expert, xperm, xsig,
+        hbuf, ypart,
         stage_x, stage_logits, stage_y, stage_switch, total;
     long long ypart_rows;  // capacity in rows of one K split
 };
@@ -129,19 +132,21 @@ void ws_layout(const dynamo_layer_desc& D, WsLayout& W) {
     W.status = take(256);
     W.counts = take(n * 4);
     W.offsets = take((n + 1) * 4);
+    W.off_pad = take((n + 1) * 4);
     W.topk_idx = take(T * k * 4);
     W.topk_w = take(T * k * 4);
     W.perm = take(T * k * 4);
     W.pos = take(T * kk * 4);
-    W.row_token = take(R * 4);
-    W.row_expert = take(R * 4);
-    W.xperm = take((R + ROW_PAD) * (d / KC) * XROW);
-    W.xsig = take((R + ROW_PAD) * std::max<size_t>(S_pad, 16) * 2);
-    W.hbuf = take((R + ROW_PAD) * (f / KC) * XROW);
+    const size_t Rp = R + 8 * n;  // physical rows: every expert's segment starts at a multiple of 8
+    W.row_token = take(Rp * 4);
+    W.row_expert = take(Rp * 4);
+    W.xperm = take((Rp + ROW_PAD) * (d / KC) * XROW);
+    W.xsig = take((Rp + ROW_PAD) * std::max<size_t>(S_pad, 16) * 2);
+    W.hbuf = take((Rp + ROW_PAD) * (f / KC) * XROW);
     const size_t ks = std::min<size_t>(MAX_KSPLIT, f / KC);
     const size_t small_rows = std::min<size_t>(R, DECODE_ROWS);
-    W.ypart_rows = (long long)std::max(R, small_rows);
-    W.ypart = take(std::max(R, ks * small_rows) * d * 4);
+    W.ypart_rows = (long long)std::max(Rp, small_rows);
+    W.ypart = take(std::max(Rp, ks * (small_rows + 8 * n)) * d * 4);
     W.stage_x = take(T * d * 2);
     W.stage_logits = take(T * (size_t)D.n_experts * 4);
     W.stage_y = take(T * d * 4);
@@ -163,6 +168,7 @@ struct dynamo_ctx {
     uint8_t* ws = nullptr;
     LayerDev host_layer;                         // host mirror of the arena header
     int switch_mode = DYNAMO_SWITCH_SELECT;
+    int tc_min_rows = TC_MIN_ROWS;               // experts with more rows take the tcgen05 path
     int64_t launches = 0;
     cudaEvent_t prof_ev[3] = {nullptr, nullptr, nullptr};  // optional: before gate/up, after gate/up, after down
     std::vector<int32_t> upload;                 // scratch for switch uploads
@@ -191,6 +197,9 @@ WsDev make_ws(const dynamo_ctx* c, int T) {
     w.R = T * (D.top_k + D.n_shared);
     w.ksplit = ksplit_for(D, T);
     w.pad_ = 0;
+    w.off_pad = (int32_t*)(b + c->W.off_pad);
+    w.Rpad = w.R + 8 * (D.n_experts + D.n_shared);
+    w.tc_min = (T > c->tc_min_rows) ? c->tc_min_rows : 0x7fffffff;  // no expert can exceed T rows
     return w;
 }
 
@@ -289,6 +298,14 @@ dynamo_status dynamo_set_profile_events(dynamo_ctx* ctx, void* before_gateup, vo
     ctx->prof_ev[0] = (cudaEvent_t)before_gateup;
     ctx->prof_ev[1] = (cudaEvent_t)after_gateup;
     ctx->prof_ev[2] = (cudaEvent_t)after_down;
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_set_tc_min_rows(dynamo_ctx* ctx, int32_t rows) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    if (rows < 0) return DYNAMO_ERR_SHAPE;
+    // the streaming path handles one 32-token chunk per expert when both paths are active
+    ctx->tc_min_rows = rows == 0 ? 0x7fffffff : (rows < TC_MIN_ROWS ? rows : TC_MIN_ROWS);
     return DYNAMO_OK;
 }
 
@@ -482,16 +499,20 @@ dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* ro
     CUDA_TRY(launch_route(router_logits, T, D.n_experts, D.top_k, D.renormalize, ws.topk_idx, ws.topk_w, st));
     CUDA_TRY(launch_scan(ws, D.n_experts, D.n_shared, D.top_k, st));
     CUDA_TRY(launch_gather(L, ws, x, st));
-    const int n_tc = (T + 31) / 32;  // an expert holds at most T rows; chunks of 32 tokens
-    const long long split_stride = (long long)ws.R * D.d_model;  // partials of one K split: [R][d]
+    const bool use_tc = ws.tc_min != 0x7fffffff;                  // experts above 32 rows take the tcgen05 path
+    const int n_tc = use_tc ? (ctx->tc_min_rows + 31) / 32 : (T + 31) / 32;                  // 32-token chunks per expert on the streaming path
+    const int n_tt = (T + 127) / 128;                             // 128-token tiles per expert on the tcgen05 path
+    const long long split_stride = (long long)ws.Rpad * D.d_model;  // partials of one K split: [Rpad][d]
     if (ctx->prof_ev[0]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[0], st));
     CUDA_TRY(launch_ffn_stream(L, ws, 1, n_tc, ctx->host_layer.n_rb13, 1, n, split_stride, FFN_SMEM_BYTES, st));
     if (ctx->prof_ev[1]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[1], st));
+    if (use_tc) CUDA_TRY(launch_ffn_tc(L, ws, 1, n_tt, ctx->host_layer.n_rb13, n, st));
     CUDA_TRY(launch_ffn_stream(L, ws, 0, n_tc, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, FFN_SMEM_BYTES,
                                st));
+    if (use_tc) CUDA_TRY(launch_ffn_tc(L, ws, 0, n_tt, ctx->host_layer.n_rb2, n, st));
     if (ctx->prof_ev[2]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[2], st));
     CUDA_TRY(launch_combine(ws, D.d_model, D.top_k, D.n_shared, y, y_dtype == DYNAMO_F32, split_stride, st));
-    ctx->launches += 6;
+    ctx->launches += use_tc ? 8 : 6;
     if (dbg) {
         const size_t tk = (size_t)T * D.top_k;
         if (dbg->topk_idx) CUDA_TRY(cudaMemcpyAsync(dbg->topk_idx, ws.topk_idx, tk * 4, cudaMemcpyDeviceToDevice, st));

@@ -61,7 +61,22 @@ struct WsDev {
     float* ypart;         // [ksplit][R][d]
     int32_t* status;      // device status word
     int32_t T, R, ksplit, pad_;
+    // Physical rows: every expert's segment starts at a multiple of 8 rows (off_pad), so that the
+    // tensor-core path can address activations as 8-row groups.  All row-indexed buffers above use
+    // physical rows; Rpad is the host-side bound R + 8 * (E + Es).
+    int32_t* off_pad;     // [E_tot + 1]
+    int32_t Rpad;
+    int32_t tc_min;       // experts with more rows than this take the tcgen05 path (INT_MAX: none)
 };
+
+// Activation layouts.  Both give a row group of 8 rows the same footprint (8 * XROW bytes per 128-k
+// chunk), so the two FFN paths can share one buffer:
+//   streaming path : row r, chunk c at (r * n_kc + c) * XROW: 128 fp16, then two fp32 sums.
+//   tcgen05 path   : row group rg, chunk c at (rg * n_kc + c) * 8 * XROW: the canonical K-major
+//                    no-swizzle MMA operand tile [k-octet 16][row 8][k 8] fp16 (2048 B).
+constexpr int TC_TILE_BYTES = 2048;
+constexpr int TC_RG_STRIDE = 8 * XROW;
+constexpr int TC_MIN_ROWS = 32;
 
 // Layers of one switch event (kernel parameter).
 struct SwitchLayers {

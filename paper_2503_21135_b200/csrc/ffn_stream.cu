@@ -22,6 +22,7 @@
 #include <type_traits>
 
 #include "common.cuh"
+#include "expand.cuh"
 #include "layout.cuh"
 
 namespace dyn {
@@ -37,96 +38,6 @@ constexpr int CHUNK_TOKENS = 32;
 __host__ __device__ inline int stage_bytes_for(int bits, int G, int NT) {
     const int b = block_bytes(bits, G) + NT * XROW;
     return (b + 127) & ~127;
-}
-
-// Packed codes of one atom for one half chunk (64 k = 4 MMA steps), per lane, plus the shifted copies.
-template <int BITS>
-struct Codes;
-template <>
-struct Codes<2> { uint32_t w[2], ws[2]; };
-template <>
-struct Codes<3> { uint32_t w[2], ws[2], t0[2], t1[2]; };
-template <>
-struct Codes<4> { uint32_t w[4], ws[4]; };
-template <>
-struct Codes<8> { uint32_t w[8]; };
-
-__device__ __forceinline__ uint32_t rotr32(uint32_t v, int n) { return __funnelshift_r(v, v, n); }
-
-template <int BITS>
-__device__ __forceinline__ void load_codes(Codes<BITS>& c, const uint8_t* atom, int lane, int half) {
-    if constexpr (BITS == 4) {
-        const uint4 v = *reinterpret_cast<const uint4*>(atom + half * 512 + lane * 16);
-        c.w[0] = v.x; c.w[1] = v.y; c.w[2] = v.z; c.w[3] = v.w;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) c.ws[i] = c.w[i] >> 8;
-    } else if constexpr (BITS == 8) {
-        const uint4 v0 = *reinterpret_cast<const uint4*>(atom + (2 * half) * 512 + lane * 16);
-        const uint4 v1 = *reinterpret_cast<const uint4*>(atom + (2 * half + 1) * 512 + lane * 16);
-        c.w[0] = v0.x; c.w[1] = v0.y; c.w[2] = v0.z; c.w[3] = v0.w;
-        c.w[4] = v1.x; c.w[5] = v1.y; c.w[6] = v1.z; c.w[7] = v1.w;
-    } else if constexpr (BITS == 2) {
-        const uint2 v = *reinterpret_cast<const uint2*>(atom + lane * 16 + half * 8);
-        c.w[0] = v.x; c.w[1] = v.y;
-        c.ws[0] = v.x >> 10; c.ws[1] = v.y >> 10;
-    } else {
-        const uint2 v = *reinterpret_cast<const uint2*>(atom + lane * 16 + half * 8);
-        const uint2 hb = *reinterpret_cast<const uint2*>(atom + 512 + lane * 8);
-        c.w[0] = v.x; c.w[1] = v.y;
-        c.ws[0] = v.x >> 8; c.ws[1] = v.y >> 8;
-        c.t0[0] = rotr32(hb.x, half * 8); c.t0[1] = rotr32(hb.y, half * 8);
-        c.t1[0] = rotr32(hb.x, half * 8 + 1); c.t1[1] = rotr32(hb.y, half * 8 + 1);
-    }
-}
-
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t r;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
-    return r;
-}
-
-// A-fragment registers of step S4 (0..3) of the loaded half chunk: fp16 pairs q * 2^(o-24).
-template <int BITS, int S4>
-__device__ __forceinline__ void expand(const Codes<BITS>& c, uint32_t (&a)[4]) {
-    if constexpr (BITS == 4) {
-        constexpr int jj = S4 >> 1;
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int phi = 2 * (S4 & 1) + h;
-#pragma unroll
-            for (int rh = 0; rh < 2; ++rh) {
-                const uint32_t src = (phi < 2) ? c.w[rh * 2 + jj] : c.ws[rh * 2 + jj];
-                a[rh + 2 * h] = src & (0x000F000Fu << (4 * (phi & 1)));
-            }
-        }
-    } else if constexpr (BITS == 8) {
-        const uint32_t w0 = c.w[(S4 >> 1) * 4 + 2 * (S4 & 1)], w1 = c.w[(S4 >> 1) * 4 + 2 * (S4 & 1) + 1];
-        a[0] = prmt(w0, 0u, 0x4140u);
-        a[1] = prmt(w0, 0u, 0x4342u);
-        a[2] = prmt(w1, 0u, 0x4140u);
-        a[3] = prmt(w1, 0u, 0x4342u);
-    } else if constexpr (BITS == 2) {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int phi = 2 * S4 + h;
-#pragma unroll
-            for (int rh = 0; rh < 2; ++rh)
-                a[rh + 2 * h] = (phi <= 4) ? (c.w[rh] & (0x00030003u << (2 * phi)))
-                                           : (c.ws[rh] & (0x00030003u << ((2 * phi - 10) & 31)));
-        }
-    } else {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int phi = 2 * S4 + h;
-            const int i = phi & 3;
-#pragma unroll
-            for (int rh = 0; rh < 2; ++rh) {
-                const uint32_t lo = (phi < 4) ? c.w[rh] : c.ws[rh];
-                const uint32_t hi = (phi < 4) ? c.t0[rh] : c.t1[rh];
-                a[rh + 2 * h] = (lo & (0x00030003u << (2 * i))) | (hi & (0x00040004u << (2 * i)));
-            }
-        }
-    }
 }
 
 struct FfnParams {
@@ -430,10 +341,10 @@ __global__ void __launch_bounds__(FFN_THREADS, 2) ffn_stream_kernel(const FfnPar
     const int tc = blockIdx.x % p.n_tc;
     const int rbs = blockIdx.x / p.n_tc;
     const int rb = rbs / p.ksplit, split = rbs % p.ksplit;
-    const int off0 = p.ws.offsets[e], off1 = p.ws.offsets[e + 1];
-    const int row0 = off0 + tc * CHUNK_TOKENS;
-    if (row0 >= off1) return;
-    const int nvalid = min(CHUNK_TOKENS, off1 - row0);
+    const int cnt = p.ws.counts[e];
+    if (cnt > p.ws.tc_min || tc * CHUNK_TOKENS >= cnt) return;  // larger experts take the tcgen05 path
+    const int row0 = p.ws.off_pad[e] + tc * CHUNK_TOKENS;       // physical rows
+    const int nvalid = min(CHUNK_TOKENS, cnt - tc * CHUNK_TOKENS);
     const ExpertDev& ex = L->ex[e];
     switch (ex.bits) {
         case 2: ffn_dispatch_tiles<2, GATEUP>(p, ex, e, rb, split, row0, nvalid, smem); break;

@@ -1,0 +1,387 @@
+// Grouped dequant-GEMM on the 5th-generation tensor cores for experts with many tokens (prefill).
+//
+// One CTA = (expert, 256-row weight block = two M=128 tiles, tile of <= 128 tokens), K over the whole
+// input axis.  Roles (320 threads):
+//   warp 8  producer : bulk async copies of the packed block and of the activation operand tile
+//                      (8-row groups, K-major no-swizzle core matrices) into a 2-stage ring.
+//   warps 0-7 dequant: expand packed codes in registers and store the dequantized fp16 weights with
+//                      tcgen05.st.16x256b straight into TENSOR MEMORY as the A operand: the packed
+//                      fragment layout (layout.cuh) is exactly that instruction's register layout, so
+//                      dequantized weights never touch shared memory.  Per register pair: one AND-OR
+//                      (1024 + q*2^o in place), one HSUB2 (exact q*2^o), one HFMA2
+//                      ((q*2^o) * (s*2^-bias) + m*2^(o-bias)): the weight s*q + m rounded ONCE to fp16,
+//                      times the power of two that the pre-scaled activations undo.
+//   warp 9  MMA      : one thread issues tcgen05.mma.kind::f16 (A from TMEM, B from shared memory,
+//                      fp32 accumulators in TMEM); tcgen05.commit releases ring slots and A buffers.
+// Gate/up: the significant-channel correction follows as extra 16-channel stages (fp16 tiles of the
+// active cached channels through ldmatrix -> tcgen05.st); epilogue = tcgen05.ld, SwiGLU, fp16 h written
+// as the down GEMM's operand tiles (pre-scaled).  Down: fp32 rows out.
+// TMEM: columns 0..255 accumulators (two M tiles x 128 tokens), 256..511 two A buffers.
+#include <type_traits>
+
+#include "common.cuh"
+#include "expand.cuh"
+#include "layout.cuh"
+
+namespace dyn {
+
+constexpr int TC_DEQ_WARPS = 8;
+constexpr int TC_THREADS = 320;
+constexpr int TC_N = 128;
+constexpr int TC_WBLK_MAX = 34816;                  // largest packed block (8-bit, G = 64)
+constexpr int TC_XTILE = 16 * TC_TILE_BYTES;        // 128 tokens x 128 k fp16
+constexpr int TC_STAGE_BYTES = TC_WBLK_MAX + TC_XTILE;
+constexpr int TC_OFF_STAGE = 256;
+constexpr int TC_SMEM_BYTES = TC_OFF_STAGE + 2 * TC_STAGE_BYTES;
+constexpr int TC_SIG_TILE_STRIDE = 528;
+constexpr uint32_t TC_TMEM_COLS = 512;
+constexpr uint32_t TC_COL_A = 256;
+
+struct TcParams {
+    const LayerDev* L;
+    WsDev ws;
+    int n_tt;  // token tiles per expert launched (grid.x = n_tt * n_rb)
+};
+
+// ---- tcgen05 wrappers ----------------------------------------------------------------------
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// K-major, no swizzle: lbo = bytes between core matrices adjacent in K, sbo = between 8-row groups.
+__device__ __forceinline__ uint64_t tc_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    return (uint64_t)((addr >> 4) & 0x3fff) | ((uint64_t)((lbo >> 4) & 0x3fff) << 16) |
+           ((uint64_t)((sbo >> 4) & 0x3fff) << 32) | (1ull << 46);
+}
+__device__ __forceinline__ void tc_mma_ts(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}" ::"r"(d),
+        "r"(a), "l"(bdesc), "r"(idesc), "r"(acc), "r"(0)
+        : "memory");
+}
+__device__ __forceinline__ void tc_st_x4(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.16x256b.x4.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(
+            taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ void tc_st_x1(uint32_t taddr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3) {
+    asm volatile("tcgen05.st.sync.aligned.16x256b.x1.b32 [%0], {%1,%2,%3,%4};" ::"r"(taddr), "r"(r0), "r"(r1), "r"(r2),
+                 "r"(r3)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_ld_x4(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+
+struct TcBars {
+    uint64_t full[2], empty[2], a_full[2], a_empty[2], d_full;
+    uint32_t tmem_base;
+    volatile int poison;
+};
+
+// In-place bit offset o of the code of (MMA step S4 of a half chunk, k pair h): see layout.cuh.
+template <int BITS>
+__host__ __device__ constexpr int code_offset(int s4, int h) {
+    const int phi = 2 * s4 + h;
+    return BITS == 2 ? (phi <= 4 ? 2 * phi : 2 * phi - 10) : BITS == 3 ? 2 * (phi & 3) : BITS == 4 ? 4 * h : 0;
+}
+
+// Dequantize one packed block stage into the A buffer: this warp's two atoms, eight MMA steps.
+template <int BITS>
+__device__ __forceinline__ void tc_dequant_stage(const uint8_t* st, uint32_t a_lanes, int atom0, int lane, int G) {
+    const int gid = lane >> 2;
+    const int ngrp = KC / G;
+    constexpr int BIAS = BITS == 2 ? 4 : (BITS == 3 ? 3 : (BITS == 4 ? 2 : 0));
+    constexpr int NOFF = BITS == 2 ? 5 : (BITS == 3 ? 4 : (BITS == 4 ? 2 : 1));   // distinct offsets 0, step, 2*step, ...
+    constexpr int OSTEP = BITS == 4 ? 4 : 2;
+    const uint32_t* prm = reinterpret_cast<const uint32_t*>(st + block_code_bytes(BITS));
+    const __half2 k1024 = __float2half2_rn(1024.f);
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
+        const int atom = atom0 + a;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            Codes<BITS> cd;
+            load_codes<BITS>(cd, st + atom * atom_bytes(BITS), lane, half);
+            const int g = (G == 64) ? half : 0;
+            __half2 S2[2], M2[2][NOFF];
+#pragma unroll
+            for (int rh = 0; rh < 2; ++rh) {
+                const int r = 16 * atom + gid + 8 * rh;
+                const uint32_t pw = prm[r * ngrp + g];
+                const __half2 pp = *reinterpret_cast<const __half2*>(&pw);
+                S2[rh] = __half2half2(__hmul(__low2half(pp), __ushort_as_half((unsigned short)((15 - BIAS) << 10))));
+#pragma unroll
+                for (int i = 0; i < NOFF; ++i)  // zero-point times 2^(o - bias), exact
+                    M2[rh][i] = __half2half2(
+                        __hmul(__high2half(pp), __ushort_as_half((unsigned short)((15 + OSTEP * i - BIAS) << 10))));
+            }
+            uint32_t regs[16];
+            auto step = [&](auto S4c) {
+                constexpr int S4 = decltype(S4c)::value;
+                uint32_t af[4];
+                expand<BITS, S4, 0x64006400u>(cd, af);
+#pragma unroll
+                for (int ri = 0; ri < 4; ++ri) {
+                    const int oi = code_offset<BITS>(S4, ri >> 1) / OSTEP;
+                    const __half2 qo = __hsub2(*reinterpret_cast<const __half2*>(&af[ri]), k1024);   // q * 2^o, exact
+                    const __half2 v = __hfma2(qo, S2[ri & 1], M2[ri & 1][oi]);
+                    af[ri] = *reinterpret_cast<const uint32_t*>(&v);
+                }
+                // fragment (rowhalf, h) -> TMEM register order of the 16x256b shape: (row, col pair)
+                regs[4 * S4 + 0] = af[0];
+                regs[4 * S4 + 1] = af[2];
+                regs[4 * S4 + 2] = af[1];
+                regs[4 * S4 + 3] = af[3];
+            };
+            step(std::integral_constant<int, 0>{});
+            step(std::integral_constant<int, 1>{});
+            step(std::integral_constant<int, 2>{});
+            step(std::integral_constant<int, 3>{});
+            tc_st_x4(a_lanes + ((uint32_t)(16 * a) << 16) + 32 * half, regs);
+        }
+    }
+}
+
+template <bool GATEUP>
+__global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const LayerDev* L = p.L;
+    const int e = L->order[blockIdx.y];
+    const int cnt = p.ws.counts[e];
+    if (cnt <= p.ws.tc_min || *p.ws.status != STATUS_OK) return;  // after an expired wait nothing new starts
+    const int tt = blockIdx.x % p.n_tt, rb = blockIdx.x / p.n_tt;
+    if (tt * TC_N >= cnt) return;
+    const int n_valid = min(TC_N, cnt - tt * TC_N);
+    const int n_rg = (n_valid + 7) >> 3;
+    const int n_mma = (n_valid + 15) & ~15;
+    const int row0 = p.ws.off_pad[e] + tt * TC_N;
+    const int rg0 = row0 >> 3;
+    const ExpertDev& ex = L->ex[e];
+    const int bits = ex.bits, G = L->G, blk_bytes = ex.blk_bytes;
+    const int K = GATEUP ? L->d : L->f;
+    const int n_kc = K / KC;
+    const int S_pad = L->S_pad;
+    const int sig_cnt = (GATEUP && ex.switchable) ? L->sig_cnt[e] : 0;
+    const int n_ss = (sig_cnt + 15) >> 4;
+    const int n_it = n_kc + n_ss;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    TcBars* B = reinterpret_cast<TcBars*>(smem);
+    uint8_t* stages = smem + TC_OFF_STAGE;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&B->full[i], 1);
+            mbar_init(&B->empty[i], 1);
+            mbar_init(&B->a_full[i], TC_DEQ_WARPS);
+            mbar_init(&B->a_empty[i], 1);
+        }
+        mbar_init(&B->d_full, 1);
+        B->poison = 0;
+        fence_barrier_init();
+    }
+    if (warp == 9) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&B->tmem_base)),
+                     "r"(TC_TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tbase = B->tmem_base;
+    volatile int* poison = &B->poison;
+    int32_t* status = p.ws.status;
+    const uint8_t* wbase = (GATEUP ? ex.w13 : ex.w2) + (size_t)rb * n_kc * blk_bytes;
+    const uint8_t* xbase = GATEUP ? p.ws.xperm : p.ws.hbuf;
+
+    if (warp == 8) {
+        // ---------------- producer ----------------
+        bool ok = true;
+        for (int it = 0; it < n_it && ok; ++it) {
+            const int s = it & 1, ph = (it >> 1) & 1;
+            uint8_t* st = stages + (size_t)s * TC_STAGE_BYTES;
+            int okl = 1;
+            if (lane == 0) okl = mbar_wait_bounded(&B->empty[s], ph ^ 1, poison, status) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, okl, 0) != 0;
+            if (!ok) break;
+            if (it < n_kc) {
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(&B->full[s], (uint32_t)(blk_bytes + n_rg * TC_TILE_BYTES));
+                    bulk_g2s(st, wbase + (size_t)it * blk_bytes, (uint32_t)blk_bytes, &B->full[s]);
+                }
+                __syncwarp();
+                if (lane < n_rg)
+                    bulk_g2s(st + TC_WBLK_MAX + lane * TC_TILE_BYTES,
+                             xbase + ((size_t)(rg0 + lane) * n_kc + it) * TC_RG_STRIDE, TC_TILE_BYTES, &B->full[s]);
+            } else {
+                const int ss = it - n_kc;
+                if (lane == 0) mbar_arrive_expect_tx(&B->full[s], (uint32_t)(16 * POOL_TILE_BYTES + n_rg * 256));
+                __syncwarp();
+                if (lane < 16) {
+                    const int pos = L->sig_pool[e * S_pad + ss * 16 + lane];
+                    bulk_g2s(st + lane * TC_SIG_TILE_STRIDE, ex.pool_hi + ((size_t)rb * (L->P + 1) + pos) * RB,
+                             POOL_TILE_BYTES, &B->full[s]);
+                }
+                if (lane < n_rg)
+                    bulk_g2s(st + TC_WBLK_MAX + lane * 256,
+                             reinterpret_cast<const uint8_t*>(p.ws.xsig) + ((size_t)(rg0 + lane) * (S_pad >> 4) + ss) * 256,
+                             256, &B->full[s]);
+            }
+        }
+        if (!ok && lane == 0) {
+            const unsigned long long t0 = globaltimer_ns();
+            while (globaltimer_ns() - t0 < 2000000ull) {
+            }
+        }
+    } else if (warp == 9) {
+        // ---------------- MMA issuer (one thread) ----------------
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | ((uint32_t)(n_mma >> 3) << 17) | (8u << 24);
+            bool ok = true;
+            for (int it = 0; it < n_it && ok; ++it) {
+                const int s = it & 1, ph = (it >> 1) & 1;
+                const uint8_t* st = stages + (size_t)s * TC_STAGE_BYTES;
+                ok = mbar_wait_bounded(&B->full[s], ph, poison, status) &&
+                     mbar_wait_bounded(&B->a_full[s], ph, poison, status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t xt = smem_u32(st + TC_WBLK_MAX);
+                if (it < n_kc) {
+#pragma unroll
+                    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                        for (int k8 = 0; k8 < 8; ++k8)
+                            tc_mma_ts(tbase + 128 * mt, tbase + TC_COL_A + 128 * s + 64 * mt + 8 * k8,
+                                      tc_desc(xt + k8 * 256, 128, TC_TILE_BYTES), idesc, (it | k8) ? 1u : 0u);
+                } else {
+#pragma unroll
+                    for (int mt = 0; mt < 2; ++mt)
+                        tc_mma_ts(tbase + 128 * mt, tbase + TC_COL_A + 128 * s + 64 * mt, tc_desc(xt, 128, 256), idesc, 1u);
+                }
+                tc_commit(&B->a_empty[s]);
+                tc_commit(&B->empty[s]);
+            }
+            tc_commit(&B->d_full);
+        }
+    } else {
+        // ---------------- dequant warps, then epilogue ----------------
+        const int q = warp & 3, mt = warp >> 2;
+        const int atom0 = 8 * mt + 2 * q;
+        const int gid = lane >> 2, tid4 = lane & 3;
+        const uint32_t my_lanes = tbase + ((uint32_t)(32 * q) << 16);
+        bool ok = true;
+        for (int it = 0; it < n_it && ok; ++it) {
+            const int s = it & 1, ph = (it >> 1) & 1;
+            const uint8_t* st = stages + (size_t)s * TC_STAGE_BYTES;
+            ok = mbar_wait_bounded(&B->full[s], ph, poison, status) &&
+                 mbar_wait_bounded(&B->a_empty[s], ph ^ 1, poison, status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a_lanes = my_lanes + TC_COL_A + 128 * s + 64 * mt;
+            if (it < n_kc) {
+                switch (bits) {
+                    case 2: tc_dequant_stage<2>(st, a_lanes, atom0, lane, G); break;
+                    case 3: tc_dequant_stage<3>(st, a_lanes, atom0, lane, G); break;
+                    case 4: tc_dequant_stage<4>(st, a_lanes, atom0, lane, G); break;
+                    default: tc_dequant_stage<8>(st, a_lanes, atom0, lane, G); break;
+                }
+            } else {
+                // significant-channel stage: fp16 tiles [slot][256 rows] -> A fragments -> TMEM
+                const int mi = lane >> 3, r = lane & 7;
+#pragma unroll
+                for (int a = 0; a < 2; ++a) {
+                    uint32_t af[4];
+                    const uint32_t addr = smem_u32(st + ((mi >> 1) * 8 + r) * TC_SIG_TILE_STRIDE +
+                                                   (16 * (atom0 + a) + (mi & 1) * 8) * 2);
+                    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                                 : "=r"(af[0]), "=r"(af[1]), "=r"(af[2]), "=r"(af[3])
+                                 : "r"(addr));
+                    tc_st_x1(a_lanes + ((uint32_t)(16 * a) << 16), af[0], af[2], af[1], af[3]);
+                }
+            }
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&B->a_full[s]);
+        }
+        if (ok) ok = mbar_wait_bounded(&B->d_full, 0, poison, status);
+        tc_fence_after();
+        if (ok) {
+            const float scl[2] = {__uint_as_float((uint32_t)(127 + x_scale_exp(bits, 8 * atom0 + gid)) << 23),
+                                  __uint_as_float((uint32_t)(127 + x_scale_exp(bits, 8 * (atom0 + 1) + gid)) << 23)};
+            const int n_kc2 = L->n_rb13;
+#pragma unroll
+            for (int a = 0; a < 2; ++a) {
+                const int atom = atom0 + a;
+                for (int cb = 0; cb * 32 < n_mma; ++cb) {
+                    uint32_t r[16];
+                    tc_ld_x4(my_lanes + ((uint32_t)(16 * a) << 16) + 128 * mt + 32 * cb, r);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            const int n = 32 * cb + 8 * j + 2 * tid4 + c;
+                            const float v0 = __uint_as_float(r[4 * j + c]), v1 = __uint_as_float(r[4 * j + 2 + c]);
+                            if (n < n_valid) {
+                                if constexpr (GATEUP) {
+                                    const float h = v0 / (1.f + expf(-v0)) * v1;
+                                    const float h16 = __half2float(__float2half_rn(h));
+                                    uint8_t* dst = p.ws.hbuf + ((size_t)(rg0 + (n >> 3)) * n_kc2 + rb) * TC_RG_STRIDE +
+                                                   atom * 128 + (n & 7) * 16 + gid * 2;
+                                    *reinterpret_cast<__half*>(dst) = __float2half_rn(h16 * scl[a]);
+                                } else {
+                                    float* yrow = p.ws.ypart + (size_t)(row0 + n) * L->d + rb * RB + atom * 16 + gid;
+                                    yrow[0] = v0;
+                                    yrow[8] = v1;
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 9) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "r"(TC_TMEM_COLS) : "memory");
+    }
+}
+
+template <bool GATEUP>
+static cudaError_t launch_tc_one(const TcParams& p, dim3 grid, cudaStream_t st) {
+    cudaError_t err =
+        cudaFuncSetAttribute(ffn_tc_kernel<GATEUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
+    if (err != cudaSuccess) return err;
+    ffn_tc_kernel<GATEUP><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(p);
+    return cudaGetLastError();
+}
+
+// n_tt: 128-token tiles per expert launched; n_rb: 256-row weight blocks; n_experts: experts in L->order.
+cudaError_t launch_ffn_tc(const LayerDev* L, const WsDev& ws, int gateup, int n_tt, int n_rb, int n_experts,
+                          cudaStream_t st) {
+    TcParams p;
+    p.L = L;
+    p.ws = ws;
+    p.n_tt = n_tt;
+    dim3 grid((unsigned)(n_tt * n_rb), (unsigned)n_experts);
+    return gateup ? launch_tc_one<true>(p, grid, st) : launch_tc_one<false>(p, grid, st);
+}
+
+}  // namespace dyn

@@ -20,10 +20,11 @@ namespace {
 
 constexpr int NOALLOC_MAX_PAIRS = DYNAMO_NOALLOC_MAX_PAIRS;  // T * k
 constexpr int NOALLOC_MAX_EXPERTS = 256;
-// counts [256] | pos [pairs] | row_token [pairs] | row_expert [pairs]
-constexpr size_t SCRATCH_INTS = 256 + 3 * (size_t)NOALLOC_MAX_PAIRS;
+// counts [256] | padded offsets [264] | pos [pairs] | row_token, row_expert [pairs + 8 * 256 padding rows]
+constexpr size_t NOALLOC_ROWS = (size_t)NOALLOC_MAX_PAIRS + 8 * NOALLOC_MAX_EXPERTS;
+constexpr size_t SCRATCH_INTS = 256 + 264 + (size_t)NOALLOC_MAX_PAIRS + 2 * NOALLOC_ROWS;
 
-// Every GPU that loads the library holds this array (about 385 KiB) until the process exits.
+// Every GPU that loads the library holds this array (about 400 KiB) until the process exits.
 static __device__ __align__(256) int32_t g_route_scratch[SCRATCH_INTS];
 
 // In host code `g_route_scratch` is only a stand-in for the symbol, not a device address: the
@@ -62,9 +63,10 @@ extern "C" dynamo_status dynamo_route_permute_static(const float* router_logits,
     cudaStream_t st = (cudaStream_t)stream;
     dyn::WsDev ws = {};
     ws.counts = scratch;
-    ws.pos = scratch + 256;
+    ws.off_pad = scratch + 256;
+    ws.pos = scratch + 256 + 264;
     ws.row_token = ws.pos + NOALLOC_MAX_PAIRS;
-    ws.row_expert = ws.row_token + NOALLOC_MAX_PAIRS;
+    ws.row_expert = ws.row_token + NOALLOC_ROWS;
     ws.offsets = expert_offsets;
     ws.topk_idx = topk_idx;
     ws.topk_w = topk_w;

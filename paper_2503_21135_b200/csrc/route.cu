@@ -3,8 +3,11 @@
 // route   : top-k of the router logits per token (ties -> lower expert index), softmax weights.
 // scan    : expert histogram -> exclusive scan -> stable counting sort of the (token, slot) pairs
 //           (token-ascending inside an expert), warp-ballot ranking: deterministic, no atomics order.
-// gather  : expert-contiguous activation rows in fp16, significant columns zeroed for switchable
-//           experts (they are served by the 8-bit path), per-64 sums, plus the gathered significant columns.
+//           Also lays the experts' segments out in PHYSICAL rows (each segment starts at a multiple of 8).
+// gather  : expert-contiguous activation rows in fp16, pre-scaled for in-place code use, significant
+//           columns zeroed for switchable experts (they are served by the 8-bit path), per-group sums,
+//           plus the gathered significant columns; written in the layout of the FFN path the row's
+//           expert takes (streaming rows, or 8-row MMA operand tiles).
 // combine : y[t] = sum_j w[t,j] * Y[pos(t,j)] + sum_shared Y[pos], fp32, fixed order.
 #include "common.cuh"
 #include "layout.cuh"
@@ -52,7 +55,7 @@ __global__ void __launch_bounds__(256) route_kernel(const float* __restrict__ lo
             const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
             if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
         }
-        // remove the winner from its owner's candidates (experts already taken are marked by index)
+        // remove the winner from its owner's candidates
 #pragma unroll
         for (int i = 0; i < 8; ++i)
             if (lane + 32 * i == bi) v[i] = -INFINITY;
@@ -70,9 +73,11 @@ __global__ void __launch_bounds__(256) route_kernel(const float* __restrict__ lo
 
 // Single CTA.  Warp w ranks the pairs of experts w, w + nwarps, ...  Pair order i = t*k + j is
 // ascending in t, and a token holds an expert at most once, so rank-by-scan-order is the stable order.
+// offsets/perm are the logical (unpadded) permutation; pos/row_token/row_expert use physical rows.
 __global__ void __launch_bounds__(1024) scan_kernel(WsDev ws, int E, int Es, int k) {
     __shared__ int s_count[MAX_EXPERTS + 1];
     __shared__ int s_off[MAX_EXPERTS + 1];
+    __shared__ int s_pad[MAX_EXPERTS + 1];
     const int T = ws.T, n_pairs = T * k;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
     const int kk = k + Es;
@@ -87,18 +92,26 @@ __global__ void __launch_bounds__(1024) scan_kernel(WsDev ws, int E, int Es, int
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-        int acc = 0;
-        for (int e = 0; e < E; ++e) { s_off[e] = acc; acc += s_count[e]; }
-        s_off[E] = acc;  // = T*k
-        for (int s = 0; s < Es; ++s) { s_count[E + s] = T; s_off[E + s + 1] = s_off[E + s] + T; }
+        int acc = 0, pad = 0;
+        for (int e = 0; e < E + Es; ++e) {
+            if (e >= E) s_count[e] = T;
+            s_off[e] = acc;
+            s_pad[e] = pad;
+            acc += s_count[e];
+            pad += (s_count[e] + 7) & ~7;
+        }
+        s_off[E + Es] = acc;
+        s_pad[E + Es] = pad;
     }
     __syncthreads();
     for (int e = threadIdx.x; e <= E + Es; e += blockDim.x) {
         ws.offsets[e] = s_off[e];
+        ws.off_pad[e] = s_pad[e];
         if (e < E + Es) ws.counts[e] = s_count[e];
     }
     for (int e = warp; e < E; e += nwarps) {
-        int run = s_off[e];
+        int run = 0;
+        const int lo = s_off[e], po = s_pad[e];
         for (int base = 0; base < n_pairs; base += 32) {
             const int i = base + lane;
             const bool hit = (i < n_pairs) && (ws.topk_idx[i] == e);
@@ -106,50 +119,65 @@ __global__ void __launch_bounds__(1024) scan_kernel(WsDev ws, int E, int Es, int
             if (hit) {
                 const int r = run + __popc(m & ((1u << lane) - 1));
                 const int t = i / k, j = i - t * k;
-                ws.perm[r] = i;
-                ws.pos[t * kk + j] = r;
-                ws.row_token[r] = t;
-                ws.row_expert[r] = e;
+                ws.perm[lo + r] = i;
+                ws.pos[t * kk + j] = po + r;
+                ws.row_token[po + r] = t;
+                ws.row_expert[po + r] = e;
             }
             run += __popc(m);
         }
+        // padding rows of this expert's segment
+        const int padded = (s_count[e] + 7) & ~7;
+        if (lane < padded - s_count[e]) {
+            ws.row_token[po + s_count[e] + lane] = -1;
+            ws.row_expert[po + s_count[e] + lane] = e;
+        }
     }
     // shared experts: every token, natural order
-    for (int i = threadIdx.x; i < Es * T; i += blockDim.x) {
-        const int s = i / T, t = i - s * T;
-        const int r = n_pairs + i;
-        ws.pos[t * kk + k + s] = r;
-        ws.row_token[r] = t;
-        ws.row_expert[r] = E + s;
+    for (int s = 0; s < Es; ++s) {
+        const int po = s_pad[E + s];
+        const int padded = (T + 7) & ~7;
+        for (int t = threadIdx.x; t < padded; t += blockDim.x) {
+            if (t < T) ws.pos[t * kk + k + s] = po + t;
+            ws.row_token[po + t] = t < T ? t : -1;
+            ws.row_expert[po + t] = E + s;
+        }
     }
 }
 
-// One CTA per sorted row; warp w converts chunks w, w+8, ...  The fp16 activations are stored
-// multiplied by 2^x_scale_exp(bits of the row's expert, k) so that the FFN kernel can use packed codes
-// in place; the per-64 sums are of the unscaled fp16 values.
+// One CTA per physical row; warp w converts chunks w, w+8, ...  The fp16 activations are stored
+// multiplied by 2^x_scale_exp(bits of the row's expert, k) so that the FFN kernels can use packed codes
+// in place; the per-group sums are of the unscaled fp16 values.
 __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict__ L, WsDev ws,
                                                      const __nv_bfloat16* __restrict__ x) {
     const int row = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (row >= ws.off_pad[L->E + L->Es]) return;
     const int t = ws.row_token[row], e = ws.row_expert[row];
+    const bool tc = ws.counts[e] > ws.tc_min;
+    if (t < 0 && !tc) return;  // padding rows matter only as zero rows of an MMA operand tile
     const int d = L->d;
+    const int n_kc = d / KC;
     const int bits = L->ex[e].bits;
     const bool sw = L->ex[e].switchable != 0;
     const uint32_t* mask = sw ? (L->sigmask + (long long)e * (d / 32)) : nullptr;
-    const __nv_bfloat16* xr = x + (long long)t * d;
-    uint8_t* out = ws.xperm + (long long)row * (d / KC) * XROW;
+    const __nv_bfloat16* xr = x + (long long)(t < 0 ? 0 : t) * d;
     const float sc0 = __uint_as_float((uint32_t)(127 + x_scale_exp(bits, 4 * lane)) << 23);
     const float sc1 = __uint_as_float((uint32_t)(127 + x_scale_exp(bits, 4 * lane + 2)) << 23);
-    for (int c = warp; c < d / KC; c += 8) {
+    const int rg = row >> 3, rr = row & 7;
+    for (int c = warp; c < n_kc; c += 8) {
         const int k0 = c * KC + lane * 4;
-        const uint2 raw = *reinterpret_cast<const uint2*>(xr + k0);
-        const __nv_bfloat162 p0 = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
-        const __nv_bfloat162 p1 = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
-        float v[4] = {__low2float(p0), __high2float(p0), __low2float(p1), __high2float(p1)};
-        if (sw) {
-            const uint32_t mw = mask[k0 >> 5] >> (k0 & 31);
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+        if (t >= 0) {
+            const uint2 raw = *reinterpret_cast<const uint2*>(xr + k0);
+            const __nv_bfloat162 p0 = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+            const __nv_bfloat162 p1 = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+            v[0] = __low2float(p0); v[1] = __high2float(p0); v[2] = __low2float(p1); v[3] = __high2float(p1);
+            if (sw) {
+                const uint32_t mw = mask[k0 >> 5] >> (k0 & 31);
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if ((mw >> i) & 1u) v[i] = 0.f;
+                for (int i = 0; i < 4; ++i)
+                    if ((mw >> i) & 1u) v[i] = 0.f;
+            }
         }
         float hv[4];
         float sum = 0.f;
@@ -165,17 +193,34 @@ __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict_
         uint2 packed;
         packed.x = *reinterpret_cast<const uint32_t*>(&oa);
         packed.y = *reinterpret_cast<const uint32_t*>(&ob);
-        *reinterpret_cast<uint2*>(out + (long long)c * XROW + lane * 8) = packed;
-        if ((lane & 15) == 0)
-            *reinterpret_cast<float*>(out + (long long)c * XROW + XROW_SUM_OFF + (lane >> 4) * 4) = sum;
+        if (!tc) {
+            uint8_t* out = ws.xperm + ((long long)row * n_kc + c) * XROW;
+            *reinterpret_cast<uint2*>(out + lane * 8) = packed;
+            if ((lane & 15) == 0) *reinterpret_cast<float*>(out + XROW_SUM_OFF + (lane >> 4) * 4) = sum;
+        } else {
+            uint8_t* out = ws.xperm + ((long long)rg * n_kc + c) * TC_RG_STRIDE;
+            *reinterpret_cast<uint2*>(out + (lane >> 1) * 128 + rr * 16 + (lane & 1) * 8) = packed;
+        }
     }
     // gathered significant columns (unscaled)
     const int S_pad = L->S_pad;
     const int cnt = sw ? L->sig_cnt[e] : 0;
     for (int j = threadIdx.x; j < S_pad; j += blockDim.x) {
-        __half hv = __float2half_rn(0.f);
-        if (j < cnt) hv = __float2half_rn(__bfloat162float(xr[L->sig_chan[e * S_pad + j]]));
-        ws.xsig[(long long)row * S_pad + j] = hv;
+        if (!tc) {
+            __half hv = __float2half_rn(0.f);
+            if (j < cnt) hv = __float2half_rn(__bfloat162float(xr[L->sig_chan[e * S_pad + j]]));
+            ws.xsig[(long long)row * S_pad + j] = hv;
+        } else {
+            // operand position kp of sub-stage ss holds slot ss*16 + sigma(kp): the A tile reaches TMEM through
+            // an ldmatrix fragment whose k pairs (2t, 2t+1 | 2t+8, 2t+9) land on TMEM k 4t .. 4t+3.
+            const int ss = j >> 4, kp = j & 15;
+            const int slot = ss * 16 + 2 * (kp >> 2) + (kp & 1) + ((kp & 2) ? 8 : 0);
+            __half hv = __float2half_rn(0.f);
+            if (t >= 0 && slot < cnt) hv = __float2half_rn(__bfloat162float(xr[L->sig_chan[e * S_pad + slot]]));
+            __half* o = reinterpret_cast<__half*>(reinterpret_cast<uint8_t*>(ws.xsig) +
+                                                  ((long long)rg * (S_pad >> 4) + ss) * 256 + (kp >> 3) * 128 + rr * 16) + (kp & 7);
+            *o = hv;
+        }
     }
 }
 
@@ -191,7 +236,8 @@ __global__ void __launch_bounds__(256) combine_kernel(WsDev ws, int d, int k, in
         const int r = ws.pos[t * kk + j];
         const float w = (j < k) ? ws.topk_w[t * k + j] : 1.0f;
         float s[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int sp = 0; sp < ws.ksplit; ++sp) {
+        const int ns = (ws.counts[ws.row_expert[r]] > ws.tc_min) ? 1 : ws.ksplit;  // the tensor-core path does not split K
+        for (int sp = 0; sp < ns; ++sp) {
             const float4 v = *reinterpret_cast<const float4*>(ws.ypart + sp * split_stride + (long long)r * d + c);
             s[0] += v.x; s[1] += v.y; s[2] += v.z; s[3] += v.w;
         }
@@ -220,12 +266,13 @@ cudaError_t launch_scan(const WsDev& ws, int E, int Es, int k, cudaStream_t st) 
     return cudaGetLastError();
 }
 cudaError_t launch_gather(const LayerDev* L, const WsDev& ws, const void* x, cudaStream_t st) {
-    gather_kernel<<<ws.R, 256, 0, st>>>(L, ws, (const __nv_bfloat16*)x);
+    gather_kernel<<<ws.Rpad, 256, 0, st>>>(L, ws, (const __nv_bfloat16*)x);
     return cudaGetLastError();
 }
 cudaError_t launch_combine(const WsDev& ws, int d, int k, int Es, void* y, int y_f32, long long split_stride,
                            cudaStream_t st) {
-    combine_kernel<<<dim3((unsigned)ws.T, (unsigned)((d + 1023) / 1024)), 256, 0, st>>>(ws, d, k, Es, y, y_f32, split_stride);
+    combine_kernel<<<dim3((unsigned)ws.T, (unsigned)((d + 1023) / 1024)), 256, 0, st>>>(ws, d, k, Es, y, y_f32,
+                                                                                       split_stride);
     return cudaGetLastError();
 }
 
