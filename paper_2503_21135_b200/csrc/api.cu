@@ -505,8 +505,8 @@ dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* ro
     const long long split_stride = (long long)ws.Rpad * D.d_model;  // partials of one K split: [Rpad][d]
     if (ctx->prof_ev[0]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[0], st));
     CUDA_TRY(launch_ffn_stream(L, ws, 1, n_tc, ctx->host_layer.n_rb13, 1, n, split_stride, FFN_SMEM_BYTES, st));
-    if (ctx->prof_ev[1]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[1], st));
     if (use_tc) CUDA_TRY(launch_ffn_tc(L, ws, 1, n_tt, ctx->host_layer.n_rb13, n, st));
+    if (ctx->prof_ev[1]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[1], st));
     CUDA_TRY(launch_ffn_stream(L, ws, 0, n_tc, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, FFN_SMEM_BYTES,
                                st));
     if (use_tc) CUDA_TRY(launch_ffn_tc(L, ws, 0, n_tt, ctx->host_layer.n_rb2, n, st));

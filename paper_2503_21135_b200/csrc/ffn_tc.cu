@@ -25,14 +25,16 @@
 
 namespace dyn {
 
-constexpr int TC_DEQ_WARPS = 8;
-constexpr int TC_THREADS = 320;
+constexpr int TC_DEQ_WARPS = 16;                    // one 16-row atom each: enough warps to hide the dequant latency
+constexpr int TC_APW = 1;                           // atoms per dequant warp
+constexpr int TC_THREADS = (TC_DEQ_WARPS + 2) * 32;
 constexpr int TC_N = 128;
 constexpr int TC_WBLK_MAX = 34816;                  // largest packed block (8-bit, G = 64)
 constexpr int TC_XTILE = 16 * TC_TILE_BYTES;        // 128 tokens x 128 k fp16
 constexpr int TC_STAGE_BYTES = TC_WBLK_MAX + TC_XTILE;
 constexpr int TC_OFF_STAGE = 256;
-constexpr int TC_SMEM_BYTES = TC_OFF_STAGE + 2 * TC_STAGE_BYTES;
+constexpr int TC_NS = 3;                            // ring depth: must cover the L2 latency of the operand tiles
+constexpr int TC_SMEM_BYTES = TC_OFF_STAGE + TC_NS * TC_STAGE_BYTES;
 constexpr int TC_SIG_TILE_STRIDE = 528;
 constexpr uint32_t TC_TMEM_COLS = 512;
 constexpr uint32_t TC_COL_A = 256;
@@ -87,7 +89,7 @@ __device__ __forceinline__ void tc_ld_x4(uint32_t taddr, uint32_t (&r)[16]) {
 }
 
 struct TcBars {
-    uint64_t full[2], empty[2], a_full[2], a_empty[2], d_full;
+    uint64_t full[TC_NS], empty[TC_NS], a_full[2], a_empty[2], d_full;
     uint32_t tmem_base;
     volatile int poison;
 };
@@ -110,7 +112,7 @@ __device__ __forceinline__ void tc_dequant_stage(const uint8_t* st, uint32_t a_l
     const uint32_t* prm = reinterpret_cast<const uint32_t*>(st + block_code_bytes(BITS));
     const __half2 k1024 = __float2half2_rn(1024.f);
 #pragma unroll
-    for (int a = 0; a < 2; ++a) {
+    for (int a = 0; a < TC_APW; ++a) {
         const int atom = atom0 + a;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -177,16 +179,18 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p)
     const int S_pad = L->S_pad;
     const int sig_cnt = (GATEUP && ex.switchable) ? L->sig_cnt[e] : 0;
     const int n_ss = (sig_cnt + 15) >> 4;
-    const int n_it = n_kc + n_ss;
+    const int n_it = n_kc + ((n_ss + 3) >> 2);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     TcBars* B = reinterpret_cast<TcBars*>(smem);
     uint8_t* stages = smem + TC_OFF_STAGE;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < TC_NS; ++i) {
             mbar_init(&B->full[i], 1);
             mbar_init(&B->empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
             mbar_init(&B->a_full[i], TC_DEQ_WARPS);
             mbar_init(&B->a_empty[i], 1);
         }
@@ -194,7 +198,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p)
         B->poison = 0;
         fence_barrier_init();
     }
-    if (warp == 9) {
+    if (warp == TC_DEQ_WARPS + 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&B->tmem_base)),
                      "r"(TC_TMEM_COLS)
                      : "memory");
@@ -209,11 +213,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p)
     const uint8_t* wbase = (GATEUP ? ex.w13 : ex.w2) + (size_t)rb * n_kc * blk_bytes;
     const uint8_t* xbase = GATEUP ? p.ws.xperm : p.ws.hbuf;
 
-    if (warp == 8) {
+    if (warp == TC_DEQ_WARPS) {
         // ---------------- producer ----------------
         bool ok = true;
         for (int it = 0; it < n_it && ok; ++it) {
-            const int s = it & 1, ph = (it >> 1) & 1;
+            const int s = it % TC_NS, ph = (it / TC_NS) & 1;  // shared-memory ring slot
+            const int b = it & 1, bph = (it >> 1) & 1;        // tensor-memory A buffer
             uint8_t* st = stages + (size_t)s * TC_STAGE_BYTES;
             int okl = 1;
             if (lane == 0) okl = mbar_wait_bounded(&B->empty[s], ph ^ 1, poison, status) ? 1 : 0;
@@ -229,18 +234,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p)
                     bulk_g2s(st + TC_WBLK_MAX + lane * TC_TILE_BYTES,
                              xbase + ((size_t)(rg0 + lane) * n_kc + it) * TC_RG_STRIDE, TC_TILE_BYTES, &B->full[s]);
             } else {
-                const int ss = it - n_kc;
-                if (lane == 0) mbar_arrive_expect_tx(&B->full[s], (uint32_t)(16 * POOL_TILE_BYTES + n_rg * 256));
+                // up to four 16-channel sub-stages (64 cached-channel tiles) per ring stage
+                const int ss0 = 4 * (it - n_kc), nsub = min(4, n_ss - ss0);
+                if (lane == 0)
+                    mbar_arrive_expect_tx(&B->full[s], (uint32_t)(nsub * 16 * POOL_TILE_BYTES + n_rg * nsub * 256));
                 __syncwarp();
-                if (lane < 16) {
-                    const int pos = L->sig_pool[e * S_pad + ss * 16 + lane];
-                    bulk_g2s(st + lane * TC_SIG_TILE_STRIDE, ex.pool_hi + ((size_t)rb * (L->P + 1) + pos) * RB,
+                for (int sl = lane; sl < nsub * 16; sl += 32) {
+                    const int pos = L->sig_pool[e * S_pad + ss0 * 16 + sl];
+                    bulk_g2s(st + sl * TC_SIG_TILE_STRIDE, ex.pool_hi + ((size_t)rb * (L->P + 1) + pos) * RB,
                              POOL_TILE_BYTES, &B->full[s]);
                 }
                 if (lane < n_rg)
-                    bulk_g2s(st + TC_WBLK_MAX + lane * 256,
-                             reinterpret_cast<const uint8_t*>(p.ws.xsig) + ((size_t)(rg0 + lane) * (S_pad >> 4) + ss) * 256,
-                             256, &B->full[s]);
+                    bulk_g2s(st + TC_WBLK_MAX + lane * 1024,
+                             reinterpret_cast<const uint8_t*>(p.ws.xsig) + ((size_t)(rg0 + lane) * (S_pad >> 4) + ss0) * 256,
+                             (uint32_t)(nsub * 256), &B->full[s]);
             }
         }
         if (!ok && lane == 0) {
@@ -248,51 +255,62 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p)
             while (globaltimer_ns() - t0 < 2000000ull) {
             }
         }
-    } else if (warp == 9) {
+    } else if (warp == TC_DEQ_WARPS + 1) {
         // ---------------- MMA issuer (one thread) ----------------
         if (lane == 0) {
             const uint32_t idesc = (1u << 4) | ((uint32_t)(n_mma >> 3) << 17) | (8u << 24);
             bool ok = true;
             for (int it = 0; it < n_it && ok; ++it) {
-                const int s = it & 1, ph = (it >> 1) & 1;
+                const int s = it % TC_NS, ph = (it / TC_NS) & 1;  // shared-memory ring slot
+            const int b = it & 1, bph = (it >> 1) & 1;        // tensor-memory A buffer
                 const uint8_t* st = stages + (size_t)s * TC_STAGE_BYTES;
                 ok = mbar_wait_bounded(&B->full[s], ph, poison, status) &&
-                     mbar_wait_bounded(&B->a_full[s], ph, poison, status);
+                     mbar_wait_bounded(&B->a_full[b], bph, poison, status);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t xt = smem_u32(st + TC_WBLK_MAX);
                 if (it < n_kc) {
+                    // One thread feeds the tensor core: keep the per-instruction work to a few integer adds
+                    // (the descriptor of MMA step k8 is the stage's descriptor plus k8 * 256 B >> 4).
+                    const uint64_t desc0 = tc_desc(xt, 128, TC_TILE_BYTES);
+                    const uint32_t a0 = tbase + TC_COL_A + 128 * b;
+                    const uint32_t first = it ? 1u : 0u;
 #pragma unroll
-                    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-                        for (int k8 = 0; k8 < 8; ++k8)
-                            tc_mma_ts(tbase + 128 * mt, tbase + TC_COL_A + 128 * s + 64 * mt + 8 * k8,
-                                      tc_desc(xt + k8 * 256, 128, TC_TILE_BYTES), idesc, (it | k8) ? 1u : 0u);
+                    for (int k8 = 0; k8 < 8; ++k8) {
+                        tc_mma_ts(tbase, a0 + 8 * k8, desc0 + (uint64_t)(16 * k8), idesc, k8 ? 1u : first);
+                        tc_mma_ts(tbase + 128, a0 + 64 + 8 * k8, desc0 + (uint64_t)(16 * k8), idesc, k8 ? 1u : first);
+                    }
                 } else {
-#pragma unroll
-                    for (int mt = 0; mt < 2; ++mt)
-                        tc_mma_ts(tbase + 128 * mt, tbase + TC_COL_A + 128 * s + 64 * mt, tc_desc(xt, 128, 256), idesc, 1u);
+                    const int nsub = min(4, n_ss - 4 * (it - n_kc));
+                    const uint64_t desc0 = tc_desc(xt, 128, 1024);
+                    const uint32_t a0 = tbase + TC_COL_A + 128 * b;
+                    for (int j = 0; j < nsub; ++j) {
+                        tc_mma_ts(tbase, a0 + 8 * j, desc0 + (uint64_t)(16 * j), idesc, 1u);
+                        tc_mma_ts(tbase + 128, a0 + 64 + 8 * j, desc0 + (uint64_t)(16 * j), idesc, 1u);
+                    }
                 }
-                tc_commit(&B->a_empty[s]);
+                tc_commit(&B->a_empty[b]);
                 tc_commit(&B->empty[s]);
             }
             tc_commit(&B->d_full);
         }
     } else {
         // ---------------- dequant warps, then epilogue ----------------
-        const int q = warp & 3, mt = warp >> 2;
-        const int atom0 = 8 * mt + 2 * q;
+        // warp -> (TMEM lane quarter q = warp % 4, M tile, which 16-lane half of the quarter)
+        const int q = warp & 3, mt = (warp >> 2) & 1, asel = warp >> 3;
+        const int atom0 = 8 * mt + 2 * q + asel;
         const int gid = lane >> 2, tid4 = lane & 3;
-        const uint32_t my_lanes = tbase + ((uint32_t)(32 * q) << 16);
+        const uint32_t my_lanes = tbase + ((uint32_t)(32 * q + 16 * asel) << 16);
         bool ok = true;
         for (int it = 0; it < n_it && ok; ++it) {
-            const int s = it & 1, ph = (it >> 1) & 1;
+            const int s = it % TC_NS, ph = (it / TC_NS) & 1;  // shared-memory ring slot
+            const int b = it & 1, bph = (it >> 1) & 1;        // tensor-memory A buffer
             const uint8_t* st = stages + (size_t)s * TC_STAGE_BYTES;
             ok = mbar_wait_bounded(&B->full[s], ph, poison, status) &&
-                 mbar_wait_bounded(&B->a_empty[s], ph ^ 1, poison, status);
+                 mbar_wait_bounded(&B->a_empty[b], bph ^ 1, poison, status);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t a_lanes = my_lanes + TC_COL_A + 128 * s + 64 * mt;
+            const uint32_t a_lanes = my_lanes + TC_COL_A + 128 * b + 64 * mt;
             if (it < n_kc) {
                 switch (bits) {
                     case 2: tc_dequant_stage<2>(st, a_lanes, atom0, lane, G); break;
@@ -303,21 +321,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p)
             } else {
                 // significant-channel stage: fp16 tiles [slot][256 rows] -> A fragments -> TMEM
                 const int mi = lane >> 3, r = lane & 7;
+                const int nsub = min(4, n_ss - 4 * (it - n_kc));
+                for (int j = 0; j < nsub; ++j) {
 #pragma unroll
-                for (int a = 0; a < 2; ++a) {
-                    uint32_t af[4];
-                    const uint32_t addr = smem_u32(st + ((mi >> 1) * 8 + r) * TC_SIG_TILE_STRIDE +
-                                                   (16 * (atom0 + a) + (mi & 1) * 8) * 2);
-                    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                                 : "=r"(af[0]), "=r"(af[1]), "=r"(af[2]), "=r"(af[3])
-                                 : "r"(addr));
-                    tc_st_x1(a_lanes + ((uint32_t)(16 * a) << 16), af[0], af[2], af[1], af[3]);
+                    for (int a = 0; a < TC_APW; ++a) {
+                        uint32_t af[4];
+                        const uint32_t addr = smem_u32(st + (j * 16 + (mi >> 1) * 8 + r) * TC_SIG_TILE_STRIDE +
+                                                       (16 * (atom0 + a) + (mi & 1) * 8) * 2);
+                        asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                                     : "=r"(af[0]), "=r"(af[1]), "=r"(af[2]), "=r"(af[3])
+                                     : "r"(addr));
+                        tc_st_x1(a_lanes + ((uint32_t)(16 * a) << 16) + 8 * j, af[0], af[2], af[1], af[3]);
+                    }
                 }
             }
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&B->a_full[s]);
+            if (lane == 0) mbar_arrive(&B->a_full[b]);
         }
         if (ok) ok = mbar_wait_bounded(&B->d_full, 0, poison, status);
         tc_fence_after();
@@ -326,7 +347,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p)
                                   __uint_as_float((uint32_t)(127 + x_scale_exp(bits, 8 * (atom0 + 1) + gid)) << 23)};
             const int n_kc2 = L->n_rb13;
 #pragma unroll
-            for (int a = 0; a < 2; ++a) {
+            for (int a = 0; a < TC_APW; ++a) {
                 const int atom = atom0 + a;
                 for (int cb = 0; cb * 32 < n_mma; ++cb) {
                     uint32_t r[16];
@@ -359,7 +380,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p)
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 9) {
+    if (warp == TC_DEQ_WARPS + 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "r"(TC_TMEM_COLS) : "memory");
     }
 }
