@@ -294,9 +294,62 @@ def run_ours(args, rank, world, device):
                              "step_gbs": v["bytes_per_step"] / (v["ms_per_step"] / 1e3) / 1e9,
                              "step_frac_of_peak": v["bytes_per_step"] / (v["ms_per_step"] / 1e3) / 1e9 / hbm_peak}
                     for t, v in results.items()}
+    if cfg.n_experts == 8 and cfg.d_model == 4096 and not args.no_switch:
+        out["switch"] = measure_switch(layers, meta, cfg, device)
     if rank == 0 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(cfg, T, args.cpu_tokens)
     return out
+
+
+def measure_switch(layers, meta, cfg, device, T=16, events=8, steps_between=8):
+    """Runtime channel switch on the stack of layers at hand (config 5 recipe: decode batch 16, every 8 steps
+    25 % of each expert's significant channels are swapped for other cached channels): steady-state step time,
+    latency of one whole switch event (all layers, one call) on the device and on the host, and its share of a step."""
+    from paper_2503_21135_b200 import binding
+
+    n = len(layers)
+    xs = [wl.activations(cfg, T, l, step=1).to(device) for l in range(n)]
+    lgs = [wl.router_logits(cfg, T, l, step=1).to(device) for l in range(n)]
+    ys = [torch.empty((T, cfg.d_model), dtype=torch.float32, device=device) for _ in range(n)]
+
+    def stack_step():
+        for l in range(n):
+            layers[l].forward(xs[l], lgs[l], binding.F32, y=ys[l])
+
+    res = {}
+    for mode_name, mode in (("select", binding.SWITCH_SELECT), ("requant", binding.SWITCH_REQUANT)):
+        cur = [m["sets"] for m in meta]
+        for l in layers:
+            l.set_switch_mode(mode)
+        binding.set_channel_switch_many(layers, cur)
+        for _ in range(5):
+            stack_step()
+        torch.cuda.synchronize()
+        dev_ms, host_ms, step_ms = [], [], []
+        for ev in range(events):
+            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            new = [wl.switch_event(cfg, meta[l]["pool"], cur[l], l, ev) for l in range(n)]
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(steps_between):
+                stack_step()
+            e1.record()
+            t0 = time.perf_counter()
+            binding.set_channel_switch_many(layers, new)
+            host_ms.append((time.perf_counter() - t0) * 1e3)
+            e2.record()
+            torch.cuda.synchronize()
+            step_ms.append(e0.elapsed_time(e1) / steps_between)
+            dev_ms.append(e1.elapsed_time(e2))
+            cur = new
+        for l in layers:
+            l.set_switch_mode(binding.SWITCH_SELECT)
+        binding.set_channel_switch_many(layers, [m["sets"] for m in meta])
+        sm, dm, hm = float(np.median(step_ms)), float(np.median(dev_ms)), float(np.median(host_ms))
+        res[mode_name] = {"layers": n, "tokens": T, "stack_step_ms": sm, "tokens_per_s": T / (sm / 1e3),
+                          "switch_event_device_ms": dm, "switch_event_host_ms": hm,
+                          "switch_fraction_of_step": dm / sm, "events": events}
+    return res
 
 
 def cpu_baseline(cfg, T, n_tokens):
@@ -366,12 +419,18 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="decode", choices=list(wl.CONFIGS))
-    ap.add_argument("--tokens", type=int, default=64)
-    ap.add_argument("--layers", type=int, default=4, help="independent layers rotated over (weights from HBM)")
+    ap.add_argument("--tokens", type=int, default=None, help="default: the workload's largest token count")
+    ap.add_argument("--layers", type=int, default=None,
+                    help="independent layers rotated over so that weights come from HBM (default 4; 16 for switch)")
+    ap.add_argument("--no-switch", action="store_true", help="skip the runtime channel-switch measurement")
     ap.add_argument("--sweep", action="store_true", help="also time the workload's other token counts")
     ap.add_argument("--cpu-tokens", type=int, default=16, help="tokens in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.tokens is None:
+        args.tokens = max(wl.CONFIGS[args.workload].tokens)
+    if args.layers is None:
+        args.layers = wl.CONFIGS[args.workload].n_layers if args.workload == "switch" else (2 if args.tokens >= 512 else 4)
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

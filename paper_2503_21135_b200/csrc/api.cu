@@ -21,8 +21,8 @@ cudaError_t launch_scan(const WsDev& ws, int E, int Es, int k, cudaStream_t st);
 cudaError_t launch_gather(const LayerDev* L, const WsDev& ws, const void* x, cudaStream_t st);
 cudaError_t launch_combine(const WsDev& ws, int d, int k, int Es, void* y, int y_f32, long long split_stride,
                            cudaStream_t st);
-cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, int n_tc, int n_rb, int ksplit,
-                              int n_experts, long long split_stride, int smem_bytes, cudaStream_t st);
+cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int ksplit, int n_experts,
+                              long long split_stride, int smem_bytes, int n_ctas, cudaStream_t st);
 cudaError_t launch_ffn_tc(const LayerDev* L, const WsDev& ws, int gateup, int n_tt, int n_rb, int n_experts,
                           cudaStream_t st);
 cudaError_t launch_switch(const SwitchLayers& layers, int n_layers, int E, const int32_t* staging, int per_layer_ints,
@@ -169,6 +169,7 @@ struct dynamo_ctx {
     LayerDev host_layer;                         // host mirror of the arena header
     int switch_mode = DYNAMO_SWITCH_SELECT;
     int tc_min_rows = TC_MIN_ROWS;               // experts with more rows take the tcgen05 path
+    int n_sms = 148;                             // SM count of the device the layer was packed on
     int64_t launches = 0;
     cudaEvent_t prof_ev[3] = {nullptr, nullptr, nullptr};  // optional: before gate/up, after gate/up, after down
     std::vector<int32_t> upload;                 // scratch for switch uploads
@@ -399,6 +400,12 @@ dynamo_status dynamo_pack_experts(dynamo_ctx* ctx, const void* w_gate, const voi
             ctx->launches += 1;
         }
     }
+    {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+            ctx->n_sms = sms;
+    }
     ctx->packed = true;
     // install the empty significant sets (sig_pool -> zero tile, sig_chan -> -1)
     std::vector<int32_t> zero_cnt(D.n_experts, 0);
@@ -504,10 +511,11 @@ dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* ro
     const int n_tt = (T + 127) / 128;                             // 128-token tiles per expert on the tcgen05 path
     const long long split_stride = (long long)ws.Rpad * D.d_model;  // partials of one K split: [Rpad][d]
     if (ctx->prof_ev[0]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[0], st));
-    CUDA_TRY(launch_ffn_stream(L, ws, 1, n_tc, ctx->host_layer.n_rb13, 1, n, split_stride, FFN_SMEM_BYTES, st));
+    const int n_ctas = 2 * ctx->n_sms;  // persistent streaming grid: two CTAs per SM
+    CUDA_TRY(launch_ffn_stream(L, ws, 1, ctx->host_layer.n_rb13, 1, n, split_stride, FFN_SMEM_BYTES, n_ctas, st));
     if (use_tc) CUDA_TRY(launch_ffn_tc(L, ws, 1, n_tt, ctx->host_layer.n_rb13, n, st));
     if (ctx->prof_ev[1]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[1], st));
-    CUDA_TRY(launch_ffn_stream(L, ws, 0, n_tc, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, FFN_SMEM_BYTES,
+    CUDA_TRY(launch_ffn_stream(L, ws, 0, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, FFN_SMEM_BYTES, n_ctas,
                                st));
     if (use_tc) CUDA_TRY(launch_ffn_tc(L, ws, 0, n_tt, ctx->host_layer.n_rb2, n, st));
     if (ctx->prof_ev[2]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[2], st));
