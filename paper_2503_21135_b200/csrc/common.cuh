@@ -167,6 +167,32 @@ __device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], 
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// ---- programmatic dependent launch -----------------------------------------------------------
+// Every kernel of a forward is launched with the programmatic-stream-serialization attribute and
+// starts with pdl_prologue(): it lets the next kernel's CTAs be scheduled early (they park in their
+// own pdl_prologue) and then waits until the preceding kernel has completed and flushed its
+// memory, so launch latency overlaps the previous kernel's tail without changing the data flow.
+__device__ __forceinline__ void pdl_prologue() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 // ---- packed-block geometry ---------------------------------------------------------------
 
 __host__ __device__ __forceinline__ int atom_bytes(int bits) { return 256 * bits; }  // 16 rows x 128 k

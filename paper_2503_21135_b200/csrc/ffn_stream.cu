@@ -289,6 +289,7 @@ __device__ __forceinline__ bool consume_dispatch(const FfnParams& p, FfnSmem* S,
 template <bool GATEUP>
 __global__ void __launch_bounds__(FFN_THREADS, 2) ffn_stream_kernel(const FfnParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
+    pdl_prologue();
     if (*p.ws.status != STATUS_OK) return;  // after an expired wait nothing new starts
     const LayerDev* L = p.L;
     FfnSmem* S = reinterpret_cast<FfnSmem*>(smem);
@@ -433,8 +434,7 @@ static cudaError_t launch_one(const FfnParams& p, int n_ctas, cudaStream_t st) {
     cudaError_t err = cudaFuncSetAttribute(ffn_stream_kernel<GATEUP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            p.smem_bytes);
     if (err != cudaSuccess) return err;
-    ffn_stream_kernel<GATEUP><<<n_ctas, FFN_THREADS, p.smem_bytes, st>>>(p);
-    return cudaGetLastError();
+    return launch_pdl(ffn_stream_kernel<GATEUP>, dim3((unsigned)n_ctas), dim3(FFN_THREADS), (size_t)p.smem_bytes, st, p);
 }
 
 // n_ctas: persistent grid size (2 per SM).

@@ -161,6 +161,7 @@ __device__ __forceinline__ void tc_dequant_stage(const uint8_t* st, uint32_t a_l
 template <bool GATEUP>
 __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p) {
     extern __shared__ __align__(1024) uint8_t smem[];
+    pdl_prologue();
     const LayerDev* L = p.L;
     const int e = L->order[blockIdx.y];
     const int cnt = p.ws.counts[e];
@@ -390,8 +391,7 @@ static cudaError_t launch_tc_one(const TcParams& p, dim3 grid, cudaStream_t st) 
     cudaError_t err =
         cudaFuncSetAttribute(ffn_tc_kernel<GATEUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
     if (err != cudaSuccess) return err;
-    ffn_tc_kernel<GATEUP><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(p);
-    return cudaGetLastError();
+    return launch_pdl(ffn_tc_kernel<GATEUP>, grid, dim3(TC_THREADS), (size_t)TC_SMEM_BYTES, st, p);
 }
 
 // n_tt: 128-token tiles per expert launched; n_rb: 256-row weight blocks; n_experts: experts in L->order.

@@ -17,6 +17,7 @@ namespace dyn {
 // One warp per token.  E <= 256: lane l holds logits l, l+32, ...
 __global__ void __launch_bounds__(256) route_kernel(const float* __restrict__ logits, int T, int E, int k, int renorm,
                                                     int32_t* __restrict__ topk_idx, float* __restrict__ topk_w) {
+    pdl_prologue();
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (warp >= T) return;
     const float* l = logits + (long long)warp * E;
@@ -78,6 +79,7 @@ __global__ void __launch_bounds__(1024) scan_kernel(WsDev ws, int E, int Es, int
     __shared__ int s_count[MAX_EXPERTS + 1];
     __shared__ int s_off[MAX_EXPERTS + 1];
     __shared__ int s_pad[MAX_EXPERTS + 1];
+    pdl_prologue();
     const int T = ws.T, n_pairs = T * k;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
     const int kk = k + Es;
@@ -150,6 +152,7 @@ __global__ void __launch_bounds__(1024) scan_kernel(WsDev ws, int E, int Es, int
 // in place; the per-group sums are of the unscaled fp16 values.
 __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict__ L, WsDev ws,
                                                      const __nv_bfloat16* __restrict__ x) {
+    pdl_prologue();
     const int row = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (row >= ws.off_pad[L->E + L->Es]) return;
     const int t = ws.row_token[row], e = ws.row_expert[row];
@@ -227,6 +230,7 @@ __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict_
 // grid (T, ceil(d / 1024)): each thread owns four output columns of one token.
 __global__ void __launch_bounds__(256) combine_kernel(WsDev ws, int d, int k, int Es, void* __restrict__ y,
                                                       int y_f32, long long split_stride) {
+    pdl_prologue();
     const int t = blockIdx.x;
     const int kk = k + Es;
     const int c = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
@@ -257,23 +261,19 @@ __global__ void __launch_bounds__(256) combine_kernel(WsDev ws, int d, int k, in
 
 cudaError_t launch_route(const float* logits, int T, int E, int k, int renorm, int32_t* idx, float* w,
                          cudaStream_t st) {
-    route_kernel<<<(T + 7) / 8, 256, 0, st>>>(logits, T, E, k, renorm, idx, w);
-    return cudaGetLastError();
+    return launch_pdl(route_kernel, dim3((unsigned)((T + 7) / 8)), dim3(256), 0, st, logits, T, E, k, renorm, idx, w);
 }
 cudaError_t launch_scan(const WsDev& ws, int E, int Es, int k, cudaStream_t st) {
     const int warps = E < 32 ? (E < 1 ? 1 : E) : 32;
-    scan_kernel<<<1, warps * 32, 0, st>>>(ws, E, Es, k);
-    return cudaGetLastError();
+    return launch_pdl(scan_kernel, dim3(1), dim3((unsigned)(warps * 32)), 0, st, ws, E, Es, k);
 }
 cudaError_t launch_gather(const LayerDev* L, const WsDev& ws, const void* x, cudaStream_t st) {
-    gather_kernel<<<ws.Rpad, 256, 0, st>>>(L, ws, (const __nv_bfloat16*)x);
-    return cudaGetLastError();
+    return launch_pdl(gather_kernel, dim3((unsigned)ws.Rpad), dim3(256), 0, st, L, ws, (const __nv_bfloat16*)x);
 }
 cudaError_t launch_combine(const WsDev& ws, int d, int k, int Es, void* y, int y_f32, long long split_stride,
                            cudaStream_t st) {
-    combine_kernel<<<dim3((unsigned)ws.T, (unsigned)((d + 1023) / 1024)), 256, 0, st>>>(ws, d, k, Es, y, y_f32,
-                                                                                       split_stride);
-    return cudaGetLastError();
+    return launch_pdl(combine_kernel, dim3((unsigned)ws.T, (unsigned)((d + 1023) / 1024)), dim3(256), 0, st, ws, d, k, Es,
+                      y, y_f32, split_stride);
 }
 
 }  // namespace dyn
