@@ -113,7 +113,7 @@ void arena_layout(const dynamo_layer_desc& D, const int32_t* bits, ArenaLayout& 
         A.q8_u[e] = take(P * f);
         A.cw_g[e] = take(P * f * 2);
         A.cw_u[e] = take(P * f * 2);
-        A.pool_hi[e] = take(n_rb13 * (P + 1) * RB * 2);
+        A.pool_hi[e] = take(n_rb13 * ((P + 31) / 32 * 32) * POOL_TILE_PITCH);
     }
     const size_t S_pad = s_pad_of(D);
     A.cache_idx = take((size_t)D.n_experts * P * 4);
@@ -141,7 +141,7 @@ void ws_layout(const dynamo_layer_desc& D, WsLayout& W) {
     W.row_token = take(Rp * 4);
     W.row_expert = take(Rp * 4);
     W.xperm = take((Rp + ROW_PAD) * (d / KC) * XROW);
-    W.xsig = take((Rp + ROW_PAD) * std::max<size_t>(S_pad, 16) * 2);
+    W.xsig = take((Rp + ROW_PAD) * std::max<size_t>(((size_t)D.cache_size + 31) / 32 * 32, 32) * 2);  // pool columns
     W.hbuf = take((Rp + ROW_PAD) * (f / KC) * XROW);
     const size_t ks = std::min<size_t>(MAX_KSPLIT, f / KC);
     const size_t small_rows = std::min<size_t>(R, DECODE_ROWS);
@@ -200,6 +200,7 @@ WsDev make_ws(const dynamo_ctx* c, int T) {
     w.pad_ = 0;
     w.off_pad = (int32_t*)(b + c->W.off_pad);
     w.Rpad = w.R + 8 * (D.n_experts + D.n_shared);
+    w.Rcap = D.max_tokens * (D.top_k + D.n_shared) + 8 * (D.n_experts + D.n_shared) + ROW_PAD;
     w.tc_min = (T > c->tc_min_rows) ? c->tc_min_rows : 0x7fffffff;  // no expert can exceed T rows
     return w;
 }
@@ -354,6 +355,7 @@ dynamo_status dynamo_pack_experts(dynamo_ctx* ctx, const void* w_gate, const voi
     std::memset(&L, 0, sizeof(L));
     L.d = d; L.f = f; L.E = D.n_experts; L.Es = D.n_shared; L.k = D.top_k; L.G = G;
     L.S = D.max_sig; L.S_pad = s_pad_of(D); L.P = P; L.renorm = D.renormalize;
+    L.P_pad = (P + 31) / 32 * 32;
     L.n_rb13 = 2 * f / RB; L.n_kc13 = d / KC; L.n_rb2 = d / RB; L.n_kc2 = f / KC;
     uint8_t* base = ctx->arena;
     L.cache_idx = (int32_t*)(base + A.cache_idx);

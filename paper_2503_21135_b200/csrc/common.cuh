@@ -35,6 +35,7 @@ struct ExpertDev {
 
 struct LayerDev {
     int32_t d, f, E, Es, k, G, S, S_pad, P, renorm;
+    int32_t P_pad;        // P rounded up to a multiple of 32 (tiles beyond P are zero)
     int32_t n_rb13, n_kc13, n_rb2, n_kc2;
     int32_t* cache_idx;   // [E][P] sorted channel indices (cache headers)
     int32_t* sig_chan;    // [E][S_pad] channel of each active slot, -1 = empty
@@ -66,6 +67,7 @@ struct WsDev {
     // physical rows; Rpad is the host-side bound R + 8 * (E + Es).
     int32_t* off_pad;     // [E_tot + 1]
     int32_t Rpad;
+    int32_t Rcap;         // rows allocated in the activation buffers (their chunk pitch)
     int32_t tc_min;       // experts with more rows than this take the tcgen05 path (INT_MAX: none)
 };
 
@@ -77,6 +79,25 @@ struct WsDev {
 constexpr int TC_TILE_BYTES = 2048;
 constexpr int TC_RG_STRIDE = 8 * XROW;
 constexpr int TC_MIN_ROWS = 32;
+
+// Activation buffers are CHUNK-MAJOR: the 128-k chunk kc of row r sits at (kc * Rcap + r) * XROW, so the
+// slice "rows r0 .. r0+n of chunk kc" that one pipeline stage needs is ONE contiguous bulk copy (many small
+// copies cost the copy engine about as much each as a large one).  Rcap = allocated rows.
+__host__ __device__ __forceinline__ size_t act_off(int kc, int row, int Rcap) {
+    return ((size_t)kc * Rcap + row) * XROW;
+}
+// Gathered activations of the cached ("pool") channels, 32 columns per group pq: (pq * Rcap + r) * 64 bytes.
+constexpr int POOL_GROUP = 32;               // cached channels per significant-channel pipeline stage
+constexpr int XPOOL_ROW = POOL_GROUP * 2;    // bytes per (row, group)
+__host__ __device__ __forceinline__ size_t xpool_off(int pq, int row, int Rcap) {
+    return ((size_t)pq * Rcap + row) * XPOOL_ROW;
+}
+// 8-bit-valued fp16 tiles of the cached channels: [row block][pool position][256 rows], 528-byte pitch
+// (the pad keeps ldmatrix rows conflict-free after a contiguous copy); P_pad = P rounded up to 32.
+constexpr int POOL_TILE_PITCH = 528;
+__host__ __device__ __forceinline__ size_t pool_tile_off(int rb, int p, int P_pad) {
+    return ((size_t)rb * P_pad + p) * POOL_TILE_PITCH;
+}
 
 // Layers of one switch event (kernel parameter).
 struct SwitchLayers {

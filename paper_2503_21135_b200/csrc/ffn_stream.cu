@@ -101,7 +101,7 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
         kc1 = (int)(((long long)(im.split + 1) * n_kc) / p.ksplit);
     }
     const int sig_cnt = (GATEUP && ex.switchable) ? L->sig_cnt[im.e] : 0;
-    const int n_ss = (sig_cnt + 15) >> 4;
+    const int n_ps = sig_cnt > 0 ? (L->P_pad >> 5) : 0;
     volatile int* poison = &S->poison;
 
     float total[2][NT8][4];
@@ -195,28 +195,33 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
     }
 
     if constexpr (GATEUP) {
-        for (int ss = 0; ss < n_ss; ++ss, ++stage_it) {
+        // cached-channel stages: the 8-bit-valued tiles of 32 pool columns times their activations (zero for
+        // channels that are not significant right now), accumulated straight into the totals
+        for (int ps = 0; ps < n_ps; ++ps, ++stage_it) {
             const int s = stage_it % NS, ph = (stage_it / NS) & 1;
             if (!mbar_wait_bounded(&S->full[s], ph, poison, p.ws.status)) return false;
             const uint8_t* st = stages + S->off[s];
-            const uint8_t* xs = st + 16 * SIG_TILE_STRIDE;
-            uint32_t b0[NT8], b1[NT8];
-#pragma unroll
-            for (int j = 0; j < NT8; ++j) {
-                b0[j] = *reinterpret_cast<const uint32_t*>(xs + (8 * j + gid) * SIG_X_STRIDE + (2 * tid4) * 2);
-                b1[j] = *reinterpret_cast<const uint32_t*>(xs + (8 * j + gid) * SIG_X_STRIDE + (2 * tid4 + 8) * 2);
-            }
+            const uint8_t* xs = st + POOL_GROUP * POOL_TILE_PITCH;
             const int mi = lane >> 3, r = lane & 7;
 #pragma unroll
-            for (int a = 0; a < 2; ++a) {
-                uint32_t af[4];
-                const uint32_t addr =
-                    smem_u32(st + ((mi >> 1) * 8 + r) * SIG_TILE_STRIDE + (16 * (atom0 + a) + (mi & 1) * 8) * 2);
-                asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                             : "=r"(af[0]), "=r"(af[1]), "=r"(af[2]), "=r"(af[3])
-                             : "r"(addr));
+            for (int ks = 0; ks < POOL_GROUP / 16; ++ks) {
+                uint32_t b0[NT8], b1[NT8];
 #pragma unroll
-                for (int j = 0; j < NT8; ++j) mma16816(total[a][j], af, b0[j], b1[j]);
+                for (int j = 0; j < NT8; ++j) {
+                    b0[j] = *reinterpret_cast<const uint32_t*>(xs + (8 * j + gid) * XPOOL_ROW + (16 * ks + 2 * tid4) * 2);
+                    b1[j] = *reinterpret_cast<const uint32_t*>(xs + (8 * j + gid) * XPOOL_ROW + (16 * ks + 2 * tid4 + 8) * 2);
+                }
+#pragma unroll
+                for (int a = 0; a < 2; ++a) {
+                    uint32_t af[4];
+                    const uint32_t addr = smem_u32(st + (16 * ks + (mi >> 1) * 8 + r) * POOL_TILE_PITCH +
+                                                   (16 * (atom0 + a) + (mi & 1) * 8) * 2);
+                    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                                 : "=r"(af[0]), "=r"(af[1]), "=r"(af[2]), "=r"(af[3])
+                                 : "r"(addr));
+#pragma unroll
+                    for (int j = 0; j < NT8; ++j) mma16816(total[a][j], af, b0[j], b1[j]);
+                }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&S->empty[s]);
@@ -255,7 +260,7 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
             uint2 ov;
             ov.x = *reinterpret_cast<const uint32_t*>(&oa);
             ov.y = *reinterpret_cast<const uint32_t*>(&ob);
-            uint8_t* dst = p.ws.hbuf + ((size_t)(im.row0 + tok) * n_rb + im.rb) * XROW;
+            uint8_t* dst = p.ws.hbuf + act_off(im.rb, im.row0 + tok, p.ws.Rcap);
             *reinterpret_cast<uint2*>(dst + lane * 8) = ov;
             if ((lane & 15) == 0) *reinterpret_cast<float*>(dst + XROW_SUM_OFF + (lane >> 4) * 4) = sum;
         }
@@ -359,7 +364,7 @@ __global__ void __launch_bounds__(FFN_THREADS, 2) ffn_stream_kernel(const FfnPar
                 kc1 = (int)(((long long)(im.split + 1) * n_kc) / p.ksplit);
             }
             const uint8_t* wbase = (GATEUP ? ex.w13 : ex.w2) + (size_t)im.rb * n_kc * blk_bytes;
-            const uint8_t* xbase = (GATEUP ? p.ws.xperm : p.ws.hbuf) + (size_t)im.row0 * n_kc * XROW;
+            const uint8_t* xbuf = GATEUP ? p.ws.xperm : p.ws.hbuf;
             for (int kc = kc0; kc < kc1 && ok; ++kc, ++it) {
                 const int s = it % NS;
                 int off = 0;
@@ -370,34 +375,33 @@ __global__ void __launch_bounds__(FFN_THREADS, 2) ffn_stream_kernel(const FfnPar
                 if (!ok) break;
                 uint8_t* st = stages + off;
                 if (lane == 0) {
+                    // two copies per stage: the packed block and the (chunk-major, hence contiguous) activation slice
                     mbar_arrive_expect_tx(&S->full[s], (uint32_t)(blk_bytes + im.nvalid * XROW));
                     bulk_g2s(st, wbase + (size_t)kc * blk_bytes, (uint32_t)blk_bytes, &S->full[s]);
+                    bulk_g2s(st + blk_bytes, xbuf + act_off(kc, im.row0, p.ws.Rcap), (uint32_t)(im.nvalid * XROW), &S->full[s]);
                 }
                 __syncwarp();
-                if (lane < im.nvalid)
-                    bulk_g2s(st + blk_bytes + lane * XROW, xbase + ((size_t)lane * n_kc + kc) * XROW, XROW, &S->full[s]);
             }
             if constexpr (GATEUP) {
-                const int sig_cnt = ex.switchable ? L->sig_cnt[im.e] : 0;
-                const int n_ss = (sig_cnt + 15) >> 4;
-                for (int ss = 0; ss < n_ss && ok; ++ss, ++it) {
+                // cached-channel stages: 32 pool columns each = one 16.9 KB tile copy + one activation copy
+                const int n_ps = (ex.switchable && L->sig_cnt[im.e] > 0) ? (L->P_pad >> 5) : 0;
+                for (int ps = 0; ps < n_ps && ok; ++ps, ++it) {
                     const int s = it % NS;
                     int off = 0;
-                    if (lane == 0) off = acquire(16 * SIG_TILE_STRIDE + ((im.nvalid + 7) & ~7) * SIG_X_STRIDE);
+                    if (lane == 0) off = acquire(POOL_GROUP * POOL_TILE_PITCH + ((im.nvalid + 7) & ~7) * XPOOL_ROW);
                     off = __shfl_sync(0xffffffffu, off, 0);
                     ok = off >= 0;
                     if (!ok) break;
                     uint8_t* st = stages + off;
-                    if (lane == 0) mbar_arrive_expect_tx(&S->full[s], (uint32_t)(16 * POOL_TILE_BYTES + im.nvalid * 32));
-                    __syncwarp();
-                    if (lane < 16) {
-                        const int pos = L->sig_pool[im.e * S_pad + ss * 16 + lane];
-                        bulk_g2s(st + lane * SIG_TILE_STRIDE, ex.pool_hi + ((size_t)im.rb * (L->P + 1) + pos) * RB,
-                                 POOL_TILE_BYTES, &S->full[s]);
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(&S->full[s], (uint32_t)(POOL_GROUP * POOL_TILE_PITCH + im.nvalid * XPOOL_ROW));
+                        bulk_g2s(st, reinterpret_cast<const uint8_t*>(ex.pool_hi) + pool_tile_off(im.rb, ps * POOL_GROUP, L->P_pad),
+                                 POOL_GROUP * POOL_TILE_PITCH, &S->full[s]);
+                        bulk_g2s(st + POOL_GROUP * POOL_TILE_PITCH,
+                                 reinterpret_cast<const uint8_t*>(p.ws.xsig) + xpool_off(ps, im.row0, p.ws.Rcap),
+                                 (uint32_t)(im.nvalid * XPOOL_ROW), &S->full[s]);
                     }
-                    if (lane < im.nvalid)
-                        bulk_g2s(st + 16 * SIG_TILE_STRIDE + lane * SIG_X_STRIDE,
-                                 p.ws.xsig + (size_t)(im.row0 + lane) * S_pad + ss * 16, 32, &S->full[s]);
+                    __syncwarp();
                 }
             }
         }

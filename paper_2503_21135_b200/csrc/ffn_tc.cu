@@ -30,7 +30,7 @@ constexpr int TC_APW = 1;                           // atoms per dequant warp
 constexpr int TC_THREADS = (TC_DEQ_WARPS + 2) * 32;
 constexpr int TC_N = 128;
 constexpr int TC_WBLK_MAX = 34816;                  // largest packed block (8-bit, G = 64)
-constexpr int TC_XTILE = 16 * TC_TILE_BYTES;        // 128 tokens x 128 k fp16
+constexpr int TC_XTILE = 16 * TC_RG_STRIDE;         // 128 tokens x 128 k fp16: 16 row-group tiles at their buffer pitch
 constexpr int TC_STAGE_BYTES = TC_WBLK_MAX + TC_XTILE;
 constexpr int TC_OFF_STAGE = 256;
 constexpr int TC_NS = 3;                            // ring depth: must cover the L2 latency of the operand tiles
@@ -177,10 +177,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p)
     const int bits = ex.bits, G = L->G, blk_bytes = ex.blk_bytes;
     const int K = GATEUP ? L->d : L->f;
     const int n_kc = K / KC;
-    const int S_pad = L->S_pad;
+    const int P_pad = L->P_pad;
     const int sig_cnt = (GATEUP && ex.switchable) ? L->sig_cnt[e] : 0;
-    const int n_ss = (sig_cnt + 15) >> 4;
-    const int n_it = n_kc + ((n_ss + 3) >> 2);
+    const int n_it = n_kc + (sig_cnt > 0 ? (P_pad + 63) >> 6 : 0);   // + cached-channel stages of 64 pool columns
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     TcBars* B = reinterpret_cast<TcBars*>(smem);
@@ -227,29 +226,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p)
             if (!ok) break;
             if (it < n_kc) {
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(&B->full[s], (uint32_t)(blk_bytes + n_rg * TC_TILE_BYTES));
+                    // two copies per stage: the packed block and the operand tile (chunk-major: contiguous)
+                    mbar_arrive_expect_tx(&B->full[s], (uint32_t)(blk_bytes + n_rg * TC_RG_STRIDE));
                     bulk_g2s(st, wbase + (size_t)it * blk_bytes, (uint32_t)blk_bytes, &B->full[s]);
+                    bulk_g2s(st + TC_WBLK_MAX, xbase + act_off(it, 8 * rg0, p.ws.Rcap), (uint32_t)(n_rg * TC_RG_STRIDE),
+                             &B->full[s]);
                 }
-                __syncwarp();
-                if (lane < n_rg)
-                    bulk_g2s(st + TC_WBLK_MAX + lane * TC_TILE_BYTES,
-                             xbase + ((size_t)(rg0 + lane) * n_kc + it) * TC_RG_STRIDE, TC_TILE_BYTES, &B->full[s]);
-            } else {
-                // up to four 16-channel sub-stages (64 cached-channel tiles) per ring stage
-                const int ss0 = 4 * (it - n_kc), nsub = min(4, n_ss - ss0);
-                if (lane == 0)
-                    mbar_arrive_expect_tx(&B->full[s], (uint32_t)(nsub * 16 * POOL_TILE_BYTES + n_rg * nsub * 256));
-                __syncwarp();
-                for (int sl = lane; sl < nsub * 16; sl += 32) {
-                    const int pos = L->sig_pool[e * S_pad + ss0 * 16 + sl];
-                    bulk_g2s(st + sl * TC_SIG_TILE_STRIDE, ex.pool_hi + ((size_t)rb * (L->P + 1) + pos) * RB,
-                             POOL_TILE_BYTES, &B->full[s]);
-                }
-                if (lane < n_rg)
-                    bulk_g2s(st + TC_WBLK_MAX + lane * 1024,
-                             reinterpret_cast<const uint8_t*>(p.ws.xsig) + ((size_t)(rg0 + lane) * (S_pad >> 4) + ss0) * 256,
-                             (uint32_t)(nsub * 256), &B->full[s]);
+            } else if (lane == 0) {
+                // cached-channel stage: up to 64 pool columns = one tile copy + one operand copy per 32 columns
+                const int c0 = 64 * (it - n_kc), ngr = min(2, (P_pad - c0) >> 5);
+                mbar_arrive_expect_tx(&B->full[s], (uint32_t)(ngr * POOL_GROUP * POOL_TILE_PITCH + ngr * n_rg * 512));
+                bulk_g2s(st, reinterpret_cast<const uint8_t*>(ex.pool_hi) + pool_tile_off(rb, c0, P_pad),
+                         (uint32_t)(ngr * POOL_GROUP * POOL_TILE_PITCH), &B->full[s]);
+                for (int g = 0; g < ngr; ++g)
+                    bulk_g2s(st + TC_WBLK_MAX + g * 8192,
+                             reinterpret_cast<const uint8_t*>(p.ws.xsig) + xpool_off((c0 >> 5) + g, 8 * rg0, p.ws.Rcap),
+                             (uint32_t)(n_rg * 512), &B->full[s]);
             }
+            __syncwarp();
         }
         if (!ok && lane == 0) {
             const unsigned long long t0 = globaltimer_ns();
@@ -273,7 +267,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p)
                 if (it < n_kc) {
                     // One thread feeds the tensor core: keep the per-instruction work to a few integer adds
                     // (the descriptor of MMA step k8 is the stage's descriptor plus k8 * 256 B >> 4).
-                    const uint64_t desc0 = tc_desc(xt, 128, TC_TILE_BYTES);
+                    const uint64_t desc0 = tc_desc(xt, 128, TC_RG_STRIDE);
                     const uint32_t a0 = tbase + TC_COL_A + 128 * b;
                     const uint32_t first = it ? 1u : 0u;
 #pragma unroll
@@ -282,12 +276,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p)
                         tc_mma_ts(tbase + 128, a0 + 64 + 8 * k8, desc0 + (uint64_t)(16 * k8), idesc, k8 ? 1u : first);
                     }
                 } else {
-                    const int nsub = min(4, n_ss - 4 * (it - n_kc));
-                    const uint64_t desc0 = tc_desc(xt, 128, 1024);
+                    const int nsub = min(4, (P_pad - 64 * (it - n_kc)) >> 4);   // 16-column MMA steps in this stage
                     const uint32_t a0 = tbase + TC_COL_A + 128 * b;
                     for (int j = 0; j < nsub; ++j) {
-                        tc_mma_ts(tbase, a0 + 8 * j, desc0 + (uint64_t)(16 * j), idesc, 1u);
-                        tc_mma_ts(tbase + 128, a0 + 64 + 8 * j, desc0 + (uint64_t)(16 * j), idesc, 1u);
+                        // operand tile of the 32-column group j/2: [row group][k-octet 4][8][8], step (j & 1) = two octets
+                        const uint64_t dsc = tc_desc(xt + (j >> 1) * 8192 + (j & 1) * 256, 128, 512);
+                        tc_mma_ts(tbase, a0 + 8 * j, dsc, idesc, 1u);
+                        tc_mma_ts(tbase + 128, a0 + 64 + 8 * j, dsc, idesc, 1u);
                     }
                 }
                 tc_commit(&B->a_empty[b]);
@@ -322,7 +317,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p)
             } else {
                 // significant-channel stage: fp16 tiles [slot][256 rows] -> A fragments -> TMEM
                 const int mi = lane >> 3, r = lane & 7;
-                const int nsub = min(4, n_ss - 4 * (it - n_kc));
+                const int nsub = min(4, (P_pad - 64 * (it - n_kc)) >> 4);
                 for (int j = 0; j < nsub; ++j) {
 #pragma unroll
                     for (int a = 0; a < TC_APW; ++a) {
@@ -364,7 +359,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ffn_tc_kernel(const TcParams p)
                                 if constexpr (GATEUP) {
                                     const float h = v0 / (1.f + expf(-v0)) * v1;
                                     const float h16 = __half2float(__float2half_rn(h));
-                                    uint8_t* dst = p.ws.hbuf + ((size_t)(rg0 + (n >> 3)) * n_kc2 + rb) * TC_RG_STRIDE +
+                                    uint8_t* dst = p.ws.hbuf + act_off(rb, 8 * (rg0 + (n >> 3)), p.ws.Rcap) +
                                                    atom * 128 + (n & 7) * 16 + gid * 2;
                                     *reinterpret_cast<__half*>(dst) = __float2half_rn(h16 * scl[a]);
                                 } else {

@@ -114,7 +114,7 @@ __global__ void pack_hi_kernel(const __nv_bfloat16* __restrict__ w_gate, const _
             const int q = quantize_code(bf16_to_double(w), s, m, HI_BITS);
             ex.pool_q8[mat][(long long)pi * f + n] = (uint8_t)q;
             ex.cache_w[mat][(long long)pi * f + n] = w;
-            ex.pool_hi[((long long)rb * (P + 1) + pi) * RB + rib] = __double2half(s * (double)q + m);
+            ex.pool_hi[pool_tile_off(rb, pi, (P + 31) & ~31) / 2 + rib] = __double2half(s * (double)q + m);
             ++pi;
         }
     }
@@ -143,7 +143,7 @@ __global__ void requant_from_cache_kernel(const LayerDev* __restrict__ L, const 
     const int q = quantize_code(bf16_to_double(w), s, m, HI_BITS);
     ex.pool_q8[mat][(long long)p * L->f + n] = (uint8_t)q;
     const int rb = n >> 7, rib = w13_row_in_block(n, mat);
-    ex.pool_hi[((long long)rb * (L->P + 1) + p) * RB + rib] = __double2half(s * (double)q + m);
+    ex.pool_hi[pool_tile_off(rb, p, L->P_pad) / 2 + rib] = __double2half(s * (double)q + m);
 }
 
 // Export logical codes and params.  One thread per (n, k).

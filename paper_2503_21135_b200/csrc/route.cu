@@ -197,32 +197,43 @@ __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict_
         packed.x = *reinterpret_cast<const uint32_t*>(&oa);
         packed.y = *reinterpret_cast<const uint32_t*>(&ob);
         if (!tc) {
-            uint8_t* out = ws.xperm + ((long long)row * n_kc + c) * XROW;
+            uint8_t* out = ws.xperm + act_off(c, row, ws.Rcap);
             *reinterpret_cast<uint2*>(out + lane * 8) = packed;
             if ((lane & 15) == 0) *reinterpret_cast<float*>(out + XROW_SUM_OFF + (lane >> 4) * 4) = sum;
         } else {
-            uint8_t* out = ws.xperm + ((long long)rg * n_kc + c) * TC_RG_STRIDE;
+            uint8_t* out = ws.xperm + act_off(c, 8 * rg, ws.Rcap);
             *reinterpret_cast<uint2*>(out + (lane >> 1) * 128 + rr * 16 + (lane & 1) * 8) = packed;
         }
     }
-    // gathered significant columns (unscaled)
-    const int S_pad = L->S_pad;
-    const int cnt = sw ? L->sig_cnt[e] : 0;
-    for (int j = threadIdx.x; j < S_pad; j += blockDim.x) {
+    // Activations of ALL cached channels of the row's expert, unscaled, zero where the channel is not
+    // currently significant: the FFN kernels multiply them with the contiguous 8-bit-valued tiles of the
+    // whole cache pool, so a switch only has to flip mask bits.
+    if (!sw) return;
+    const int P = L->P, P_pad = L->P_pad;
+    const int32_t* ci = L->cache_idx + (long long)e * P;
+    uint8_t* xp = reinterpret_cast<uint8_t*>(ws.xsig);
+    for (int j = threadIdx.x; j < P_pad; j += blockDim.x) {
+        const int pq = j >> 5, col = j & 31;
         if (!tc) {
-            __half hv = __float2half_rn(0.f);
-            if (j < cnt) hv = __float2half_rn(__bfloat162float(xr[L->sig_chan[e * S_pad + j]]));
-            ws.xsig[(long long)row * S_pad + j] = hv;
+            float v = 0.f;
+            if (j < P) {
+                const int ch = ci[j];
+                if ((mask[ch >> 5] >> (ch & 31)) & 1u) v = __bfloat162float(xr[ch]);
+            }
+            *reinterpret_cast<__half*>(xp + xpool_off(pq, row, ws.Rcap) + col * 2) = __float2half_rn(v);
         } else {
-            // operand position kp of sub-stage ss holds slot ss*16 + sigma(kp): the A tile reaches TMEM through
-            // an ldmatrix fragment whose k pairs (2t, 2t+1 | 2t+8, 2t+9) land on TMEM k 4t .. 4t+3.
-            const int ss = j >> 4, kp = j & 15;
-            const int slot = ss * 16 + 2 * (kp >> 2) + (kp & 1) + ((kp & 2) ? 8 : 0);
-            __half hv = __float2half_rn(0.f);
-            if (t >= 0 && slot < cnt) hv = __float2half_rn(__bfloat162float(xr[L->sig_chan[e * S_pad + slot]]));
-            __half* o = reinterpret_cast<__half*>(reinterpret_cast<uint8_t*>(ws.xsig) +
-                                                  ((long long)rg * (S_pad >> 4) + ss) * 256 + (kp >> 3) * 128 + rr * 16) + (kp & 7);
-            *o = hv;
+            // operand position kp of a 16-column step holds pool column 16*step + sigma(kp): the A tile reaches
+            // TMEM through an ldmatrix fragment whose k pairs (2t, 2t+1 | 2t+8, 2t+9) land on TMEM k 4t .. 4t+3.
+            const int step = col >> 4, kp = col & 15;
+            const int pj = pq * 32 + step * 16 + 2 * (kp >> 2) + (kp & 1) + ((kp & 2) ? 8 : 0);
+            float v = 0.f;
+            if (t >= 0 && pj < P) {
+                const int ch = ci[pj];
+                if ((mask[ch >> 5] >> (ch & 31)) & 1u) v = __bfloat162float(xr[ch]);
+            }
+            // 8-row operand tile of group pq: [k-octet 4][row 8][8 k] fp16 = 512 B
+            *reinterpret_cast<__half*>(xp + xpool_off(pq, 8 * rg, ws.Rcap) + (col >> 3) * 128 + rr * 16 + (col & 7) * 2) =
+                __float2half_rn(v);
         }
     }
 }
