@@ -22,7 +22,7 @@ cudaError_t launch_gather(const LayerDev* L, const WsDev& ws, const void* x, cud
 cudaError_t launch_combine(const WsDev& ws, int d, int k, int Es, void* y, int y_f32, long long split_stride,
                            cudaStream_t st);
 cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int ksplit, int n_experts,
-                              long long split_stride, int smem_bytes, int n_ctas, cudaStream_t st);
+                              long long split_stride, int max_rows, int n_sms, cudaStream_t st);
 cudaError_t launch_ffn_tc(const LayerDev* L, const WsDev& ws, int gateup, int n_tt, int n_rb, int n_experts,
                           cudaStream_t st);
 cudaError_t launch_switch(const SwitchLayers& layers, int n_layers, int E, const int32_t* staging, int per_layer_ints,
@@ -513,12 +513,11 @@ dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* ro
     const int n_tt = (T + 127) / 128;                             // 128-token tiles per expert on the tcgen05 path
     const long long split_stride = (long long)ws.Rpad * D.d_model;  // partials of one K split: [Rpad][d]
     if (ctx->prof_ev[0]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[0], st));
-    const int n_ctas = 2 * ctx->n_sms;  // persistent streaming grid: two CTAs per SM
-    CUDA_TRY(launch_ffn_stream(L, ws, 1, ctx->host_layer.n_rb13, 1, n, split_stride, FFN_SMEM_BYTES, n_ctas, st));
+    const int max_rows = use_tc ? std::min(T, ctx->tc_min_rows) : T;  // rows one expert can have on the streaming path
+    CUDA_TRY(launch_ffn_stream(L, ws, 1, ctx->host_layer.n_rb13, 1, n, split_stride, max_rows, ctx->n_sms, st));
     if (use_tc) CUDA_TRY(launch_ffn_tc(L, ws, 1, n_tt, ctx->host_layer.n_rb13, n, st));
     if (ctx->prof_ev[1]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[1], st));
-    CUDA_TRY(launch_ffn_stream(L, ws, 0, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, FFN_SMEM_BYTES, n_ctas,
-                               st));
+    CUDA_TRY(launch_ffn_stream(L, ws, 0, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, max_rows, ctx->n_sms, st));
     if (use_tc) CUDA_TRY(launch_ffn_tc(L, ws, 0, n_tt, ctx->host_layer.n_rb2, n, st));
     if (ctx->prof_ev[2]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[2], st));
     CUDA_TRY(launch_combine(ws, D.d_model, D.top_k, D.n_shared, y, y_dtype == DYNAMO_F32, split_stride, st));

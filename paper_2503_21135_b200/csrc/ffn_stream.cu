@@ -44,6 +44,7 @@ struct FfnParams {
     long long split_stride;  // elements between K-split partial outputs
     int smem_bytes;
     int ring_bytes;          // bytes of the stage ring (stages take what they need, in order)
+    int htile_bytes;         // bytes of one h tile behind the ring
     int n_rb;                // 256-row weight blocks of the matrix
     int n_experts;
 };
@@ -230,7 +231,7 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
 
     if constexpr (GATEUP) {
         // SwiGLU: rows 0..7 of an atom are gate, rows 8..15 the matching up rows.
-        uint8_t* htile = htiles + (item_idx & 1) * (CHUNK_TOKENS * XROW);
+        uint8_t* htile = htiles + (item_idx & 1) * p.htile_bytes;
 #pragma unroll
         for (int a = 0; a < 2; ++a)
 #pragma unroll
@@ -281,18 +282,25 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
     return true;
 }
 
-template <int BITS, bool GATEUP>
+// MAXNT8: most 8-token tiles an item can have in this launch (the host knows the token count): the small
+// variants need fewer registers and run three CTAs per SM.
+template <int BITS, bool GATEUP, int MAXNT8>
 __device__ __forceinline__ bool consume_dispatch(const FfnParams& p, FfnSmem* S, uint8_t* stages, uint8_t* htiles,
                                                  const Item& im, int& stage_it, int item_idx) {
     const int nt8 = (im.nvalid + 7) >> 3;
-    if (nt8 == 1) return consume_item<BITS, 1, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
-    if (nt8 == 2) return consume_item<BITS, 2, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
-    if (nt8 == 3) return consume_item<BITS, 3, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
-    return consume_item<BITS, 4, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
+    if (MAXNT8 == 1 || nt8 == 1) return consume_item<BITS, 1, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
+    if constexpr (MAXNT8 >= 2) {
+        if (MAXNT8 == 2 || nt8 == 2) return consume_item<BITS, 2, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
+    }
+    if constexpr (MAXNT8 >= 4) {
+        if (nt8 == 3) return consume_item<BITS, 3, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
+        return consume_item<BITS, 4, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
+    }
+    return false;
 }
 
-template <bool GATEUP>
-__global__ void __launch_bounds__(FFN_THREADS, 2) ffn_stream_kernel(const FfnParams p) {
+template <bool GATEUP, int MAXNT8>
+__global__ void __launch_bounds__(FFN_THREADS, MAXNT8 <= 2 ? 3 : 2) ffn_stream_kernel(const FfnParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     pdl_prologue();
     if (*p.ws.status != STATUS_OK) return;  // after an expired wait nothing new starts
@@ -421,10 +429,10 @@ __global__ void __launch_bounds__(FFN_THREADS, 2) ffn_stream_kernel(const FfnPar
         const Item im = decode_item(p, S, g, y);
         bool ok;
         switch (L->ex[im.e].bits) {
-            case 2: ok = consume_dispatch<2, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx); break;
-            case 3: ok = consume_dispatch<3, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx); break;
-            case 4: ok = consume_dispatch<4, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx); break;
-            default: ok = consume_dispatch<8, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx); break;
+            case 2: ok = consume_dispatch<2, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx); break;
+            case 3: ok = consume_dispatch<3, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx); break;
+            case 4: ok = consume_dispatch<4, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx); break;
+            default: ok = consume_dispatch<8, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx); break;
         }
         if (!ok) {  // poisoned: the status word says so; keep arriving so that nobody waits on this warp forever
             if (GATEUP && lane == 0) mbar_arrive(&S->done);
@@ -433,27 +441,37 @@ __global__ void __launch_bounds__(FFN_THREADS, 2) ffn_stream_kernel(const FfnPar
     }
 }
 
-template <bool GATEUP>
+template <bool GATEUP, int MAXNT8>
 static cudaError_t launch_one(const FfnParams& p, int n_ctas, cudaStream_t st) {
-    cudaError_t err = cudaFuncSetAttribute(ffn_stream_kernel<GATEUP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           p.smem_bytes);
+    cudaError_t err = cudaFuncSetAttribute(ffn_stream_kernel<GATEUP, MAXNT8>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, p.smem_bytes);
     if (err != cudaSuccess) return err;
-    return launch_pdl(ffn_stream_kernel<GATEUP>, dim3((unsigned)n_ctas), dim3(FFN_THREADS), (size_t)p.smem_bytes, st, p);
+    return launch_pdl(ffn_stream_kernel<GATEUP, MAXNT8>, dim3((unsigned)n_ctas), dim3(FFN_THREADS), (size_t)p.smem_bytes,
+                      st, p);
 }
 
-// n_ctas: persistent grid size (2 per SM).
+// max_rows: upper bound of the rows one expert can have in this forward (selects the kernel variant);
+// n_sms: SM count (the persistent grid is 2 or 3 CTAs per SM).
 cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int ksplit, int n_experts,
-                              long long split_stride, int smem_bytes, int n_ctas, cudaStream_t st) {
+                              long long split_stride, int max_rows, int n_sms, cudaStream_t st) {
+    // three CTAs per SM pay off once every CTA has several items to walk; at 1-3 tokens a CTA sees one or two
+    const bool small = max_rows >= 4 && max_rows <= 16;
+    const int smem_bytes = small ? 74 * 1024 : 110 * 1024;
+    const int n_ctas = (small ? 3 : 2) * n_sms;
     FfnParams p;
     p.L = L;
     p.ws = ws;
     p.ksplit = ksplit;
     p.split_stride = split_stride;
     p.smem_bytes = smem_bytes;
-    p.ring_bytes = (smem_bytes - SMEM_HEADER - (gateup ? 2 * CHUNK_TOKENS * XROW : 0)) & ~127;
+    // two h tiles (double-buffered across items) behind the ring; the small variants hold at most 16 tokens
+    p.htile_bytes = (small ? 16 : CHUNK_TOKENS) * XROW;
+    p.ring_bytes = (smem_bytes - SMEM_HEADER - (gateup ? 2 * p.htile_bytes : 0)) & ~127;
     p.n_rb = n_rb;
     p.n_experts = n_experts;
-    return gateup ? launch_one<true>(p, n_ctas, st) : launch_one<false>(p, n_ctas, st);
+    if (small && max_rows <= 8) return gateup ? launch_one<true, 1>(p, n_ctas, st) : launch_one<false, 1>(p, n_ctas, st);
+    if (small) return gateup ? launch_one<true, 2>(p, n_ctas, st) : launch_one<false, 2>(p, n_ctas, st);
+    return gateup ? launch_one<true, 4>(p, n_ctas, st) : launch_one<false, 4>(p, n_ctas, st);
 }
 
 }  // namespace dyn
