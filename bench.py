@@ -98,7 +98,7 @@ class ClockSampler:
         return out
 
 
-def build_layers(cfg, n_layers, max_tokens, device):
+def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None):
     """Generate, upload and pack ``n_layers`` independent layers; they share one workspace."""
     from paper_2503_21135_b200 import binding
 
@@ -111,6 +111,8 @@ def build_layers(cfg, n_layers, max_tokens, device):
         layer = binding.DynamoLayer.from_config(cfg, max_tokens=max_tokens, workspace=ws, device=device)
         layer.pack_experts(wg.to(device), wu.to(device), wd.to(device), bits, pool)
         layer.set_channel_switch(sets)
+        if tc_min_rows is not None:
+            layer.set_tc_min_rows(tc_min_rows)
         torch.cuda.synchronize()
         ws = layer.workspace
         layers.append(layer)
@@ -177,7 +179,7 @@ def run_ours(args, rank, world, device):
         if world > 1:
             torch.distributed.barrier()
 
-    layers, meta = build_layers(cfg, n_layers, max(T, max(cfg.tokens)), device)
+    layers, meta = build_layers(cfg, n_layers, max(T, max(cfg.tokens)), device, args.tc_min_rows)
     sweep_T = sorted(set([T] + (list(cfg.tokens) if args.sweep else [])))
     results = {}
     for Tcur in sweep_T:
@@ -423,6 +425,8 @@ def main():
     ap.add_argument("--layers", type=int, default=None,
                     help="independent layers rotated over so that weights come from HBM (default 4; 16 for switch)")
     ap.add_argument("--no-switch", action="store_true", help="skip the runtime channel-switch measurement")
+    ap.add_argument("--tc-min-rows", type=int, default=None,
+                    help="experts with more rows than this take the tcgen05 kernel (0: streaming kernel only)")
     ap.add_argument("--sweep", action="store_true", help="also time the workload's other token counts")
     ap.add_argument("--cpu-tokens", type=int, default=16, help="tokens in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -23,7 +23,7 @@ cudaError_t launch_combine(const WsDev& ws, int d, int k, int Es, void* y, int y
                            cudaStream_t st);
 cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int ksplit, int n_experts,
                               long long split_stride, int max_rows, int n_sms, cudaStream_t st);
-cudaError_t launch_ffn_tc(const LayerDev* L, const WsDev& ws, int gateup, int n_tt, int n_rb, int n_experts,
+cudaError_t launch_ffn_tc(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int n_experts, int n_sms,
                           cudaStream_t st);
 cudaError_t launch_switch(const SwitchLayers& layers, int n_layers, int E, const int32_t* staging, int per_layer_ints,
                           cudaStream_t st);
@@ -36,7 +36,6 @@ namespace {
 constexpr size_t ALIGN = 256;
 constexpr int ROW_PAD = 32;            // extra activation rows so a token chunk may read past the last row
 constexpr int MAX_SWITCH_LAYERS = 64;
-constexpr int FFN_SMEM_BYTES = 110 * 1024;
 constexpr int DECODE_ROWS = 1024;      // up to this many permuted rows the down GEMM is split along K
 constexpr int MAX_KSPLIT = 8;
 
@@ -201,7 +200,9 @@ WsDev make_ws(const dynamo_ctx* c, int T) {
     w.off_pad = (int32_t*)(b + c->W.off_pad);
     w.Rpad = w.R + 8 * (D.n_experts + D.n_shared);
     w.Rcap = D.max_tokens * (D.top_k + D.n_shared) + 8 * (D.n_experts + D.n_shared) + ROW_PAD;
-    w.tc_min = (T > c->tc_min_rows) ? c->tc_min_rows : 0x7fffffff;  // no expert can exceed T rows
+    // No expert can exceed T rows.  Up to twice the threshold the streaming kernel takes a large expert as
+    // two 32-token chunks (the second pass over its blocks hits L2), which costs less than two more launches.
+    w.tc_min = (c->tc_min_rows != 0x7fffffff && T > 2 * c->tc_min_rows) ? c->tc_min_rows : 0x7fffffff;
     return w;
 }
 
@@ -509,16 +510,14 @@ dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* ro
     CUDA_TRY(launch_scan(ws, D.n_experts, D.n_shared, D.top_k, st));
     CUDA_TRY(launch_gather(L, ws, x, st));
     const bool use_tc = ws.tc_min != 0x7fffffff;                  // experts above 32 rows take the tcgen05 path
-    const int n_tc = use_tc ? (ctx->tc_min_rows + 31) / 32 : (T + 31) / 32;                  // 32-token chunks per expert on the streaming path
-    const int n_tt = (T + 127) / 128;                             // 128-token tiles per expert on the tcgen05 path
     const long long split_stride = (long long)ws.Rpad * D.d_model;  // partials of one K split: [Rpad][d]
     if (ctx->prof_ev[0]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[0], st));
     const int max_rows = use_tc ? std::min(T, ctx->tc_min_rows) : T;  // rows one expert can have on the streaming path
     CUDA_TRY(launch_ffn_stream(L, ws, 1, ctx->host_layer.n_rb13, 1, n, split_stride, max_rows, ctx->n_sms, st));
-    if (use_tc) CUDA_TRY(launch_ffn_tc(L, ws, 1, n_tt, ctx->host_layer.n_rb13, n, st));
+    if (use_tc) CUDA_TRY(launch_ffn_tc(L, ws, 1, ctx->host_layer.n_rb13, n, ctx->n_sms, st));
     if (ctx->prof_ev[1]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[1], st));
     CUDA_TRY(launch_ffn_stream(L, ws, 0, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, max_rows, ctx->n_sms, st));
-    if (use_tc) CUDA_TRY(launch_ffn_tc(L, ws, 0, n_tt, ctx->host_layer.n_rb2, n, st));
+    if (use_tc) CUDA_TRY(launch_ffn_tc(L, ws, 0, ctx->host_layer.n_rb2, n, ctx->n_sms, st));
     if (ctx->prof_ev[2]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[2], st));
     CUDA_TRY(launch_combine(ws, D.d_model, D.top_k, D.n_shared, y, y_dtype == DYNAMO_F32, split_stride, st));
     ctx->launches += use_tc ? 8 : 6;

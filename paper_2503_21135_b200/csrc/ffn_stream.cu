@@ -31,8 +31,6 @@ namespace dyn {
 
 constexpr int CONSUMER_WARPS = 8;
 constexpr int FFN_THREADS = (CONSUMER_WARPS + 1) * 32;
-constexpr int SIG_TILE_STRIDE = 528;  // 512 B tile + 16 B pad: conflict-free ldmatrix rows
-constexpr int SIG_X_STRIDE = 48;      // 32 B of gathered activations per token + pad
 constexpr int SMEM_HEADER = 2048;     // barriers, poison flag, per-expert item prefix table
 constexpr int MAX_STAGES = 16;        // ring queue depth; the ring itself is byte-granular
 constexpr int CHUNK_TOKENS = 32;
@@ -246,7 +244,6 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
         __syncwarp();
         if (lane == 0) mbar_arrive(&S->done);
         if (!mbar_wait_bounded(&S->done, item_idx & 1, poison, p.ws.status)) return false;
-        const int n_rb = L->n_rb13;  // = chunks of the hidden axis
         // this lane's four hidden indices 4*lane + {0..3}: the down matrix wants them scaled by 2^(bias-o)
         const float sc0 = __uint_as_float((uint32_t)(127 + x_scale_exp(BITS, 4 * lane)) << 23);
         const float sc1 = __uint_as_float((uint32_t)(127 + x_scale_exp(BITS, 4 * lane + 2)) << 23);
@@ -361,7 +358,6 @@ __global__ void __launch_bounds__(FFN_THREADS, MAXNT8 <= 2 ? 3 : 2) ffn_stream_k
         };
         const int K = GATEUP ? L->d : L->f;
         const int n_kc = K / KC;
-        const int S_pad = L->S_pad;
         for (int g = blockIdx.x; g < n_items && ok; g += gridDim.x) {
             const Item im = decode_item(p, S, g, y);
             const ExpertDev& ex = L->ex[im.e];

@@ -72,10 +72,16 @@ __global__ void __launch_bounds__(256) route_kernel(const float* __restrict__ lo
     }
 }
 
-// Single CTA.  Warp w ranks the pairs of experts w, w + nwarps, ...  Pair order i = t*k + j is
-// ascending in t, and a token holds an expert at most once, so rank-by-scan-order is the stable order.
+// Single CTA of 32 warps.  The pair array (pair i = t*k + j, ascending in t) is cut into 32 contiguous
+// segments, one per warp.  Pass 1: each warp histograms its segment per expert (lanes holding the same
+// expert find one another with match.any; the lowest lane of each group adds the group's size).
+// An exclusive scan over segments turns the histograms into each segment's first rank within the
+// expert; pass 2 walks the segment again and ranks each pair = segment base + pairs of that expert
+// seen so far in the segment + position within the 32-pair batch.  Segments and lanes ascend in i and
+// a token holds an expert at most once, so the rank is the stable order.
 // offsets/perm are the logical (unpadded) permutation; pos/row_token/row_expert use physical rows.
 __global__ void __launch_bounds__(1024) scan_kernel(WsDev ws, int E, int Es, int k) {
+    __shared__ int s_hist[32][MAX_EXPERTS];
     __shared__ int s_count[MAX_EXPERTS + 1];
     __shared__ int s_off[MAX_EXPERTS + 1];
     __shared__ int s_pad[MAX_EXPERTS + 1];
@@ -83,27 +89,59 @@ __global__ void __launch_bounds__(1024) scan_kernel(WsDev ws, int E, int Es, int
     const int T = ws.T, n_pairs = T * k;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
     const int kk = k + Es;
-    for (int e = warp; e < E; e += nwarps) {
-        int c = 0;
-        for (int base = 0; base < n_pairs; base += 32) {
-            const int i = base + lane;
-            const bool hit = (i < n_pairs) && (ws.topk_idx[i] == e);
-            c += __popc(__ballot_sync(0xffffffffu, hit));
-        }
-        if (lane == 0) s_count[e] = c;
+    const int per_warp = ((n_pairs + 31) / 32 + nwarps - 1) / nwarps * 32;  // whole 32-pair batches per segment
+    const int seg_lo = min(n_pairs, warp * per_warp), seg_hi = min(n_pairs, seg_lo + per_warp);
+    const unsigned lt = (1u << lane) - 1;
+    for (int e = lane; e < E; e += 32) s_hist[warp][e] = 0;
+    __syncwarp();
+    for (int base = seg_lo; base < seg_hi; base += 32) {
+        const int i = base + lane;
+        const bool valid = i < seg_hi;
+        const int e = valid ? ws.topk_idx[i] : -1;
+        const unsigned m = __match_any_sync(0xffffffffu, e);
+        if (valid && (m & lt) == 0) s_hist[warp][e] += __popc(m);
+        __syncwarp();
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        int acc = 0, pad = 0;
-        for (int e = 0; e < E + Es; ++e) {
-            if (e >= E) s_count[e] = T;
-            s_off[e] = acc;
-            s_pad[e] = pad;
-            acc += s_count[e];
-            pad += (s_count[e] + 7) & ~7;
+    for (int e = threadIdx.x; e < E + Es; e += blockDim.x) {
+        int acc = 0;
+        if (e < E) {
+            for (int w = 0; w < nwarps; ++w) {
+                const int c = s_hist[w][e];
+                s_hist[w][e] = acc;
+                acc += c;
+            }
+        } else {
+            acc = T;
         }
-        s_off[E + Es] = acc;
-        s_pad[E + Es] = pad;
+        s_count[e] = acc;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int run = 0, run_pad = 0;
+        for (int e0 = 0; e0 < E + Es; e0 += 32) {
+            const int e = e0 + lane;
+            const int c = e < E + Es ? s_count[e] : 0;
+            int v = c, vp = (c + 7) & ~7;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int u = __shfl_up_sync(0xffffffffu, v, d), up = __shfl_up_sync(0xffffffffu, vp, d);
+                if (lane >= d) {
+                    v += u;
+                    vp += up;
+                }
+            }
+            if (e < E + Es) {
+                s_off[e] = run + v - c;
+                s_pad[e] = run_pad + vp - ((c + 7) & ~7);
+            }
+            run += __shfl_sync(0xffffffffu, v, 31);
+            run_pad += __shfl_sync(0xffffffffu, vp, 31);
+        }
+        if (lane == 0) {
+            s_off[E + Es] = run;
+            s_pad[E + Es] = run_pad;
+        }
     }
     __syncthreads();
     for (int e = threadIdx.x; e <= E + Es; e += blockDim.x) {
@@ -111,28 +149,31 @@ __global__ void __launch_bounds__(1024) scan_kernel(WsDev ws, int E, int Es, int
         ws.off_pad[e] = s_pad[e];
         if (e < E + Es) ws.counts[e] = s_count[e];
     }
-    for (int e = warp; e < E; e += nwarps) {
-        int run = 0;
-        const int lo = s_off[e], po = s_pad[e];
-        for (int base = 0; base < n_pairs; base += 32) {
-            const int i = base + lane;
-            const bool hit = (i < n_pairs) && (ws.topk_idx[i] == e);
-            const unsigned m = __ballot_sync(0xffffffffu, hit);
-            if (hit) {
-                const int r = run + __popc(m & ((1u << lane) - 1));
-                const int t = i / k, j = i - t * k;
-                ws.perm[lo + r] = i;
-                ws.pos[t * kk + j] = po + r;
-                ws.row_token[po + r] = t;
-                ws.row_expert[po + r] = e;
-            }
-            run += __popc(m);
+    for (int base = seg_lo; base < seg_hi; base += 32) {
+        const int i = base + lane;
+        const bool valid = i < seg_hi;
+        const int e = valid ? ws.topk_idx[i] : -1;
+        const unsigned m = __match_any_sync(0xffffffffu, e);
+        const int start = valid ? s_hist[warp][e] : 0;
+        __syncwarp();
+        if (valid && (m & lt) == 0) s_hist[warp][e] = start + __popc(m);
+        __syncwarp();
+        if (valid) {
+            const int r = start + __popc(m & lt);
+            const int t = i / k, j = i - t * k;
+            const int po = s_pad[e];
+            ws.perm[s_off[e] + r] = i;
+            ws.pos[t * kk + j] = po + r;
+            ws.row_token[po + r] = t;
+            ws.row_expert[po + r] = e;
         }
-        // padding rows of this expert's segment
-        const int padded = (s_count[e] + 7) & ~7;
-        if (lane < padded - s_count[e]) {
-            ws.row_token[po + s_count[e] + lane] = -1;
-            ws.row_expert[po + s_count[e] + lane] = e;
+    }
+    // padding rows of each routed expert's segment
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+        const int c = s_count[e], po = s_pad[e];
+        for (int r = c; r < ((c + 7) & ~7); ++r) {
+            ws.row_token[po + r] = -1;
+            ws.row_expert[po + r] = e;
         }
     }
     // shared experts: every token, natural order
@@ -275,7 +316,8 @@ cudaError_t launch_route(const float* logits, int T, int E, int k, int renorm, i
     return launch_pdl(route_kernel, dim3((unsigned)((T + 7) / 8)), dim3(256), 0, st, logits, T, E, k, renorm, idx, w);
 }
 cudaError_t launch_scan(const WsDev& ws, int E, int Es, int k, cudaStream_t st) {
-    const int warps = E < 32 ? (E < 1 ? 1 : E) : 32;
+    const int batches = (ws.T * k + 31) / 32;  // one warp per segment of whole 32-pair batches
+    const int warps = batches < 8 ? 8 : (batches > 32 ? 32 : batches);  // >= 8: the per-expert loops want threads
     return launch_pdl(scan_kernel, dim3(1), dim3((unsigned)(warps * 32)), 0, st, ws, E, Es, k);
 }
 cudaError_t launch_gather(const LayerDev* L, const WsDev& ws, const void* x, cudaStream_t st) {

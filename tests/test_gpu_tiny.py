@@ -78,6 +78,31 @@ def test_forward_parity_and_routing(tiny, T):
     assert err <= TOL, err
 
 
+@pytest.mark.parametrize("T", [40, 64, 200])
+def test_tensor_core_and_streaming_kernels_agree_with_the_oracle(tiny, T):
+    """The same tokens through either FFN kernel: experts above 8 rows on the tcgen05 kernel, then
+    every expert on the streaming kernel (large experts as 32-token chunks)."""
+    gpu = tiny["gpu"]
+    out = {}
+    try:
+        for rows in (8, 0):
+            gpu.set_tc_min_rows(rows)
+            y, _, ref, _, _ = _forward_both(tiny, T, tiny["sets"], step=300 + T)
+            assert rel_err(y, ref["y"]) <= TOL, (rows, rel_err(y, ref["y"]))
+            out[rows] = y
+    finally:
+        gpu.set_tc_min_rows(32)
+    assert np.max(np.abs(out[8] - out[0])) <= TOL * np.sqrt(np.mean(out[0].astype(np.float64) ** 2))
+    launches = []
+    for rows in (8, 0):   # the two settings really take different paths: 8 vs 6 kernels per forward
+        gpu.set_tc_min_rows(rows)
+        n0 = gpu.kernel_launches()
+        _forward_both(tiny, T, tiny["sets"], step=300 + T)
+        launches.append(gpu.kernel_launches() - n0)
+    gpu.set_tc_min_rows(32)
+    assert launches[0] - launches[1] == 2, launches
+
+
 def test_empty_sets_and_bf16_output(tiny):
     empty = [np.zeros((0,), np.int32)] * CFG.n_experts
     y, _, ref, x, lg = _forward_both(tiny, 64, empty, step=1)
