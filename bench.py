@@ -142,7 +142,7 @@ def time_steps(fn, steps, dist_barrier):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one gate/up launch, from the ncu captures summarised
 # under profiles/ (decode shape, layer 0); None where no capture of that launch exists.
-NCU_TRAFFIC_BYTES = {("decode", 8): 466.4e6 + 4.4e6}
+NCU_TRAFFIC_BYTES = {("decode", 8): 466.4e6 + 4.4e6, ("decode", 64): 498.1e6 + 13.3e6}
 
 
 def kernel_times(layers, step_fn, steps):
@@ -163,6 +163,20 @@ def kernel_times(layers, step_fn, steps):
     gu = [evs[i][0].elapsed_time(evs[i][1]) for i in range(n)]
     dn = [evs[i][1].elapsed_time(evs[i][2]) for i in range(n)]
     return float(np.mean(gu)), float(np.mean(dn))
+
+
+def slowest_rank(times_ms, world, device):
+    """Replicas only: ranks exchange nothing but their timings; a job is as slow as its slowest rank."""
+    if world <= 1:
+        return list(times_ms)
+    t = torch.tensor(list(times_ms), device=device, dtype=torch.float64)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def job_throughput(tokens_per_rank, world, ms_per_step):
+    """Whole-job tokens/s: every rank pushes its own batch through its own replica (weak scaling)."""
+    return world * tokens_per_rank / (ms_per_step / 1e3)
 
 
 def run_ours(args, rank, world, device):
@@ -242,12 +256,9 @@ def run_ours(args, rank, world, device):
 
     r = results[T]
     ms_step = r["ms_per_step"]
-    if world > 1:
-        t = torch.tensor([ms_step, ms_e2e], device=device, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms_step, ms_e2e = float(t[0]), float(t[1])
-    value = world * T / (ms_step / 1e3)
-    e2e_value = world * T / (ms_e2e / args.steps / 1e3)
+    ms_step, ms_e2e = slowest_rank([ms_step, ms_e2e], world, device)
+    value = job_throughput(T, world, ms_step)
+    e2e_value = job_throughput(T, world, ms_e2e / args.steps)
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

@@ -1,0 +1,55 @@
+"""The N > 1 path of bench.py on CPU: ranks are independent replicas (no data-path collective), the only
+exchange is the MAX of their timings; the reference arm runs on rank 0 alone."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+
+def _rank_main(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+
+    mine = [1.0 + rank, 10.0 - 3 * rank]           # rank 0: (1, 10); rank 1: (2, 7)
+    got = bench.slowest_rank(mine, world, torch.device("cpu"))
+    with open(os.path.join(out_dir, f"r{rank}.json"), "w") as f:
+        json.dump(got, f)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_timings_reduce_to_the_slowest_rank_world2(tmp_path):
+    port = 29500 + os.getpid() % 2000
+    mp.spawn(_rank_main, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    for r in range(2):
+        assert json.load(open(tmp_path / f"r{r}.json")) == [2.0, 10.0]
+
+
+def test_job_throughput_is_the_sum_over_replicas():
+    import bench
+
+    assert bench.slowest_rank([3.0, 4.0], 1, torch.device("cpu")) == [3.0, 4.0]
+    assert bench.job_throughput(64, 1, 0.5) == pytest.approx(128000.0)
+    assert bench.job_throughput(64, 8, 0.5) == pytest.approx(8 * 128000.0)
+
+
+def test_reference_arm_runs_on_rank0_only():
+    env = dict(os.environ, WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT="29999")
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--workload", "tiny",
+           "--steps", "1", "--warmup", "0", "--cpu-tokens", "4"]
+    r1 = subprocess.run(cmd, env=dict(env, RANK="1", LOCAL_RANK="1"), capture_output=True, text=True, timeout=300)
+    assert r1.returncode == 0 and r1.stdout.strip() == ""
+    r0 = subprocess.run(cmd, env=dict(env, RANK="0", LOCAL_RANK="0"), capture_output=True, text=True, timeout=300)
+    assert r0.returncode == 0, r0.stderr[-2000:]
+    line = json.loads(r0.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["cpu_baseline"]["kind"] == "oracle"

@@ -1,6 +1,7 @@
 """Pins for the CPU oracle: every function is checked against something other than itself
 (a library routine, a closed form, an invariant, brute force on tiny inputs)."""
 import itertools
+import os
 
 import numpy as np
 import pytest
@@ -158,12 +159,19 @@ def test_pack_roundtrip(bits, K):
 
 
 def test_pack_bit_positions_hand_example():
-    # 3-bit codes 1..7,0,... : code k sits at bits [3k, 3k+3) of a little-endian stream.
-    q = np.array([[1, 2, 3, 4, 5, 6, 7, 0, 1, 2, 3, 4]], dtype=np.uint8)  # 36 bits -> 2 words
-    words = oracle.pack_rows(q, 3)
-    stream = sum(int(c) << (3 * k) for k, c in enumerate(q[0]))
-    assert int(words[0, 0]) == stream & 0xFFFFFFFF and int(words[0, 1]) == stream >> 32
-    assert int(words[0, 0]) == 0xD11F58D1 and int(words[0, 1]) == 0x8
+    # hand-worked fixture: code k sits at bits [3k, 3k+3) of a little-endian stream
+    fx = {}
+    for line in open(os.path.join(os.path.dirname(__file__), "golden", "pack_3bit_words.txt")):
+        if line.strip() and not line.startswith("#"):
+            key, *vals = line.split()
+            fx[key] = vals
+    bits = int(fx["bits"][0])
+    q = np.array([[int(v) for v in fx["codes"]]], dtype=np.uint8)
+    expect = [int(v, 16) for v in fx["words"]]
+    words = oracle.pack_rows(q, bits)
+    assert [int(w) for w in words[0]] == expect
+    stream = sum(int(c) << (bits * k) for k, c in enumerate(q[0]))
+    assert expect[0] == stream & 0xFFFFFFFF and expect[1] == stream >> 32
 
 
 def test_groups_stay_word_aligned():
