@@ -98,7 +98,7 @@ class ClockSampler:
         return out
 
 
-def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None):
+def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None, decode_kernel=None):
     """Generate, upload and pack ``n_layers`` independent layers; they share one workspace."""
     from paper_2503_21135_b200 import binding
 
@@ -113,6 +113,8 @@ def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None):
         layer.set_channel_switch(sets)
         if tc_min_rows is not None:
             layer.set_tc_min_rows(tc_min_rows)
+        if decode_kernel is not None:
+            layer.set_decode_kernel(binding.DECODE_STREAM if decode_kernel == "stream" else binding.DECODE_TENSOR)
         torch.cuda.synchronize()
         ws = layer.workspace
         layers.append(layer)
@@ -193,7 +195,7 @@ def run_ours(args, rank, world, device):
         if world > 1:
             torch.distributed.barrier()
 
-    layers, meta = build_layers(cfg, n_layers, max(T, max(cfg.tokens)), device, args.tc_min_rows)
+    layers, meta = build_layers(cfg, n_layers, max(T, max(cfg.tokens)), device, args.tc_min_rows, args.decode_kernel)
     sweep_T = sorted(set([T] + (list(cfg.tokens) if args.sweep else [])))
     results = {}
     for Tcur in sweep_T:
@@ -297,7 +299,9 @@ def run_ours(args, rank, world, device):
     if T < 512:
       out["roofline"] = {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                        "frac": achieved / hbm_peak, "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, T)),
-                       "peak_kind": peak_kind, "kernel": "ffn_stream_kernel<gate/up>",
+                       "peak_kind": peak_kind,
+                       "kernel": "ffn_tcd_kernel<gate/up>" if (args.decode_kernel == "tensor" and T <= 64)
+                       else "ffn_stream_kernel<gate/up>",
                        "algorithmic_bytes_per_launch": r["gu_bytes"], "avg_launch_ms": r["gu_ms"],
                        "down_launch": {"achieved": r["dn_bytes"] / (r["dn_ms"] / 1e3) / 1e9, "avg_launch_ms": r["dn_ms"]},
                        "whole_step": {"achieved": r["bytes_per_step"] / (ms_step / 1e3) / 1e9,
@@ -438,6 +442,8 @@ def main():
     ap.add_argument("--no-switch", action="store_true", help="skip the runtime channel-switch measurement")
     ap.add_argument("--tc-min-rows", type=int, default=None,
                     help="experts with more rows than this take the tcgen05 kernel (0: streaming kernel only)")
+    ap.add_argument("--decode-kernel", default=None, choices=["tensor", "stream"],
+                    help="kernel for batches of up to 64 tokens (default: the library's, stream)")
     ap.add_argument("--sweep", action="store_true", help="also time the workload's other token counts")
     ap.add_argument("--cpu-tokens", type=int, default=16, help="tokens in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")

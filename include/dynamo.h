@@ -176,6 +176,19 @@ dynamo_status dynamo_poll_status(dynamo_ctx* ctx, void* stream);
  * 0 switches the tcgen05 path off.  Both paths implement the same arithmetic definition. */
 dynamo_status dynamo_set_tc_min_rows(dynamo_ctx* ctx, int32_t rows);
 
+/* Which kernel serves small batches (forwards of at most 64 tokens, where every expert has few rows and the
+ * forward is bound by streaming the packed weights of Section V-B from HBM):
+ *   DYNAMO_DECODE_STREAM (default): the streaming kernel (mma.sync) takes every expert, as it does for the
+ *       experts of up to 32 rows of larger batches;
+ *   DYNAMO_DECODE_TENSOR: the decode tensor-core kernel takes every expert: codes are expanded in place into
+ *       tensor memory, tcgen05.mma accumulates one quantization group at a time, scale and zero are applied
+ *       once per group when the group is read back.  Measured slower than the streaming kernel on B200
+ *       (the expand -> MMA -> fold hand-offs per 128-k stage cost more than they save); kept selectable.
+ * Both implement the same arithmetic definition.  Host-side setting; takes effect at the next forward.
+ * Errors: NULL ctx -> ERR_NULL; unknown kind -> ERR_SHAPE. */
+enum { DYNAMO_DECODE_TENSOR = 0, DYNAMO_DECODE_STREAM = 1 };
+dynamo_status dynamo_set_decode_kernel(dynamo_ctx* ctx, int32_t kind);
+
 /* Measurement hook: three cudaEvent_t handles (any may be NULL) that every following forward records on
  * its stream before the gate/up FFN launch, after it, and after the down FFN launch, so that a
  * harness can time the dominant kernels in place.  Pass NULLs to switch it off. */

@@ -25,6 +25,8 @@ cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, in
                               long long split_stride, int max_rows, int n_sms, cudaStream_t st);
 cudaError_t launch_ffn_tc(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int n_experts, int n_sms,
                           cudaStream_t st);
+cudaError_t launch_ffn_tcd(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int ksplit, int n_experts,
+                           long long split_stride, int n_sms, cudaStream_t st);
 cudaError_t launch_switch(const SwitchLayers& layers, int n_layers, int E, const int32_t* staging, int per_layer_ints,
                           cudaStream_t st);
 }  // namespace dyn
@@ -38,6 +40,7 @@ constexpr int ROW_PAD = 32;            // extra activation rows so a token chunk
 constexpr int MAX_SWITCH_LAYERS = 64;
 constexpr int DECODE_ROWS = 1024;      // up to this many permuted rows the down GEMM is split along K
 constexpr int MAX_KSPLIT = 8;
+constexpr int DECODE_FOLD_TOKENS = 64;  // up to this many tokens the decode tensor-core kernel serves every expert
 
 inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
 
@@ -168,6 +171,7 @@ struct dynamo_ctx {
     LayerDev host_layer;                         // host mirror of the arena header
     int switch_mode = DYNAMO_SWITCH_SELECT;
     int tc_min_rows = TC_MIN_ROWS;               // experts with more rows take the tcgen05 path
+    int decode_kernel = DYNAMO_DECODE_STREAM;     // which kernel serves forwards of up to DECODE_FOLD_TOKENS tokens
     int n_sms = 148;                             // SM count of the device the layer was packed on
     int64_t launches = 0;
     cudaEvent_t prof_ev[3] = {nullptr, nullptr, nullptr};  // optional: before gate/up, after gate/up, after down
@@ -196,7 +200,9 @@ WsDev make_ws(const dynamo_ctx* c, int T) {
     w.T = T;
     w.R = T * (D.top_k + D.n_shared);
     w.ksplit = ksplit_for(D, T);
-    w.pad_ = 0;
+    // Small batches: every expert has few rows, the forward is bound by streaming weights, and all experts
+    // go through the decode tensor-core kernel (operand-tile activation layout everywhere).
+    w.fold = (c->decode_kernel == DYNAMO_DECODE_TENSOR && T <= DECODE_FOLD_TOKENS) ? 1 : 0;
     w.off_pad = (int32_t*)(b + c->W.off_pad);
     w.Rpad = w.R + 8 * (D.n_experts + D.n_shared);
     w.Rcap = D.max_tokens * (D.top_k + D.n_shared) + 8 * (D.n_experts + D.n_shared) + ROW_PAD;
@@ -309,6 +315,13 @@ dynamo_status dynamo_set_tc_min_rows(dynamo_ctx* ctx, int32_t rows) {
     if (rows < 0) return DYNAMO_ERR_SHAPE;
     // the streaming path handles one 32-token chunk per expert when both paths are active
     ctx->tc_min_rows = rows == 0 ? 0x7fffffff : (rows < TC_MIN_ROWS ? rows : TC_MIN_ROWS);
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_set_decode_kernel(dynamo_ctx* ctx, int32_t kind) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    if (kind != DYNAMO_DECODE_TENSOR && kind != DYNAMO_DECODE_STREAM) return DYNAMO_ERR_SHAPE;
+    ctx->decode_kernel = kind;
     return DYNAMO_OK;
 }
 
@@ -492,6 +505,21 @@ dynamo_status dynamo_set_channel_switch(dynamo_ctx* ctx, const int32_t* sig_idx,
     return dynamo_set_channel_switch_many(one, 1, sig_idx, sig_cnt, stream);
 }
 
+// Optional copies of the routing intermediates for parity tests.
+static dynamo_status forward_debug_copies(const dynamo_ctx* ctx, const WsDev& ws, int32_t T, const dynamo_debug_out* dbg,
+                                          cudaStream_t st) {
+    if (!dbg) return DYNAMO_OK;
+    const dynamo_layer_desc& D = ctx->D;
+    const size_t tk = (size_t)T * D.top_k;
+    if (dbg->topk_idx) CUDA_TRY(cudaMemcpyAsync(dbg->topk_idx, ws.topk_idx, tk * 4, cudaMemcpyDeviceToDevice, st));
+    if (dbg->topk_w) CUDA_TRY(cudaMemcpyAsync(dbg->topk_w, ws.topk_w, tk * 4, cudaMemcpyDeviceToDevice, st));
+    if (dbg->expert_offsets)
+        CUDA_TRY(cudaMemcpyAsync(dbg->expert_offsets, ws.offsets, (size_t)(D.n_experts + 1) * 4,
+                                 cudaMemcpyDeviceToDevice, st));
+    if (dbg->perm) CUDA_TRY(cudaMemcpyAsync(dbg->perm, ws.perm, tk * 4, cudaMemcpyDeviceToDevice, st));
+    return DYNAMO_OK;
+}
+
 dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* router_logits, int32_t T, void* y,
                                  int32_t y_dtype, const dynamo_debug_out* dbg, void* stream) {
     if (!ctx) return DYNAMO_ERR_NULL;
@@ -511,6 +539,16 @@ dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* ro
     CUDA_TRY(launch_gather(L, ws, x, st));
     const bool use_tc = ws.tc_min != 0x7fffffff;                  // experts above 32 rows take the tcgen05 path
     const long long split_stride = (long long)ws.Rpad * D.d_model;  // partials of one K split: [Rpad][d]
+    if (ws.fold) {
+        if (ctx->prof_ev[0]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[0], st));
+        CUDA_TRY(launch_ffn_tcd(L, ws, 1, ctx->host_layer.n_rb13, 1, n, split_stride, ctx->n_sms, st));
+        if (ctx->prof_ev[1]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[1], st));
+        CUDA_TRY(launch_ffn_tcd(L, ws, 0, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, ctx->n_sms, st));
+        if (ctx->prof_ev[2]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[2], st));
+        CUDA_TRY(launch_combine(ws, D.d_model, D.top_k, D.n_shared, y, y_dtype == DYNAMO_F32, split_stride, st));
+        ctx->launches += 6;
+        return forward_debug_copies(ctx, ws, T, dbg, st);
+    }
     if (ctx->prof_ev[0]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[0], st));
     const int max_rows = use_tc ? std::min(T, ctx->tc_min_rows) : T;  // rows one expert can have on the streaming path
     CUDA_TRY(launch_ffn_stream(L, ws, 1, ctx->host_layer.n_rb13, 1, n, split_stride, max_rows, ctx->n_sms, st));
@@ -521,16 +559,7 @@ dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* ro
     if (ctx->prof_ev[2]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[2], st));
     CUDA_TRY(launch_combine(ws, D.d_model, D.top_k, D.n_shared, y, y_dtype == DYNAMO_F32, split_stride, st));
     ctx->launches += use_tc ? 8 : 6;
-    if (dbg) {
-        const size_t tk = (size_t)T * D.top_k;
-        if (dbg->topk_idx) CUDA_TRY(cudaMemcpyAsync(dbg->topk_idx, ws.topk_idx, tk * 4, cudaMemcpyDeviceToDevice, st));
-        if (dbg->topk_w) CUDA_TRY(cudaMemcpyAsync(dbg->topk_w, ws.topk_w, tk * 4, cudaMemcpyDeviceToDevice, st));
-        if (dbg->expert_offsets)
-            CUDA_TRY(cudaMemcpyAsync(dbg->expert_offsets, ws.offsets, (size_t)(D.n_experts + 1) * 4,
-                                     cudaMemcpyDeviceToDevice, st));
-        if (dbg->perm) CUDA_TRY(cudaMemcpyAsync(dbg->perm, ws.perm, tk * 4, cudaMemcpyDeviceToDevice, st));
-    }
-    return DYNAMO_OK;
+    return forward_debug_copies(ctx, ws, T, dbg, st);
 }
 
 dynamo_status dynamo_moe_forward_host(dynamo_ctx* ctx, const void* x_host, const float* logits_host, int32_t T,

@@ -61,7 +61,8 @@ struct WsDev {
     uint8_t* hbuf;        // [R + pad][f/128][XROW]
     float* ypart;         // [ksplit][R][d]
     int32_t* status;      // device status word
-    int32_t T, R, ksplit, pad_;
+    int32_t T, R, ksplit;
+    int32_t fold;         // 1: every expert goes through the decode tensor-core kernel (operand-tile layout everywhere)
     // Physical rows: every expert's segment starts at a multiple of 8 rows (off_pad), so that the
     // tensor-core path can address activations as 8-row groups.  All row-indexed buffers above use
     // physical rows; Rpad is the host-side bound R + 8 * (E + Es).
@@ -150,13 +151,18 @@ constexpr unsigned long long WAIT_LIMIT_NS = 1000ull * 1000ull * 1000ull;
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* poison,
                                                   int32_t* status) {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = globaltimer_ns();
+    // The clock is read only every 1024 failed polls (a poll itself suspends for a while in hardware):
+    // reading %globaltimer on every wait that does not pass at once costs far more than the wait.
+    unsigned long long t0 = 0;
     uint32_t spins = 0;
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 0xff) == 0) {
+        if ((++spins & 0x3ff) == 0) {
             if (*poison) return false;
-            if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+            const unsigned long long now = globaltimer_ns();
+            if (t0 == 0) {
+                t0 = now;
+            } else if (now - t0 > WAIT_LIMIT_NS) {
                 *poison = 1;
                 atomicExch(status, STATUS_TIMEOUT);
                 return false;

@@ -197,7 +197,7 @@ __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict_
     const int row = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (row >= ws.off_pad[L->E + L->Es]) return;
     const int t = ws.row_token[row], e = ws.row_expert[row];
-    const bool tc = ws.counts[e] > ws.tc_min;
+    const bool tc = ws.fold || ws.counts[e] > ws.tc_min;
     if (t < 0 && !tc) return;  // padding rows matter only as zero rows of an MMA operand tile
     const int d = L->d;
     const int n_kc = d / KC;
@@ -244,6 +244,8 @@ __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict_
         } else {
             uint8_t* out = ws.xperm + act_off(c, 8 * rg, ws.Rcap);
             *reinterpret_cast<uint2*>(out + (lane >> 1) * 128 + rr * 16 + (lane & 1) * 8) = packed;
+            // sums of the unscaled values per half chunk, beside the tile: [half 2][row 8] fp32
+            if ((lane & 15) == 0) *reinterpret_cast<float*>(out + TC_TILE_BYTES + ((lane >> 4) * 8 + rr) * 4) = sum;
         }
     }
     // Activations of ALL cached channels of the row's expert, unscaled, zero where the channel is not
@@ -292,7 +294,7 @@ __global__ void __launch_bounds__(256) combine_kernel(WsDev ws, int d, int k, in
         const int r = ws.pos[t * kk + j];
         const float w = (j < k) ? ws.topk_w[t * k + j] : 1.0f;
         float s[4] = {0.f, 0.f, 0.f, 0.f};
-        const int ns = (ws.counts[ws.row_expert[r]] > ws.tc_min) ? 1 : ws.ksplit;  // the tensor-core path does not split K
+        const int ns = (!ws.fold && ws.counts[ws.row_expert[r]] > ws.tc_min) ? 1 : ws.ksplit;  // the tensor-core path does not split K
         for (int sp = 0; sp < ns; ++sp) {
             const float4 v = *reinterpret_cast<const float4*>(ws.ypart + sp * split_stride + (long long)r * d + c);
             s[0] += v.x; s[1] += v.y; s[2] += v.z; s[3] += v.w;
