@@ -98,7 +98,7 @@ class ClockSampler:
         return out
 
 
-def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None, decode_kernel=None):
+def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None, decode_kernel=None, prefill_kernel=None):
     """Generate, upload and pack ``n_layers`` independent layers; they share one workspace."""
     from paper_2503_21135_b200 import binding
 
@@ -113,6 +113,8 @@ def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None, decode_ker
         layer.set_channel_switch(sets)
         if tc_min_rows is not None:
             layer.set_tc_min_rows(tc_min_rows)
+        if prefill_kernel is not None:
+            layer.set_prefill_kernel(binding.PREFILL_SINGLE if prefill_kernel == "single" else binding.PREFILL_PAIR)
         if decode_kernel is not None:
             layer.set_decode_kernel(binding.DECODE_STREAM if decode_kernel == "stream" else binding.DECODE_TENSOR)
         torch.cuda.synchronize()
@@ -195,7 +197,7 @@ def run_ours(args, rank, world, device):
         if world > 1:
             torch.distributed.barrier()
 
-    layers, meta = build_layers(cfg, n_layers, max(T, max(cfg.tokens)), device, args.tc_min_rows, args.decode_kernel)
+    layers, meta = build_layers(cfg, n_layers, max(T, max(cfg.tokens)), device, args.tc_min_rows, args.decode_kernel, args.prefill_kernel)
     sweep_T = sorted(set([T] + (list(cfg.tokens) if args.sweep else [])))
     results = {}
     for Tcur in sweep_T:
@@ -442,6 +444,8 @@ def main():
     ap.add_argument("--no-switch", action="store_true", help="skip the runtime channel-switch measurement")
     ap.add_argument("--tc-min-rows", type=int, default=None,
                     help="experts with more rows than this take the tcgen05 kernel (0: streaming kernel only)")
+    ap.add_argument("--prefill-kernel", default=None, choices=["pair", "single"],
+                    help="tcgen05 kernel for experts above the row threshold (default: the library's, pair)")
     ap.add_argument("--decode-kernel", default=None, choices=["tensor", "stream"],
                     help="kernel for batches of up to 64 tokens (default: the library's, stream)")
     ap.add_argument("--sweep", action="store_true", help="also time the workload's other token counts")

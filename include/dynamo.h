@@ -189,6 +189,16 @@ dynamo_status dynamo_set_tc_min_rows(dynamo_ctx* ctx, int32_t rows);
 enum { DYNAMO_DECODE_TENSOR = 0, DYNAMO_DECODE_STREAM = 1 };
 dynamo_status dynamo_set_decode_kernel(dynamo_ctx* ctx, int32_t kind);
 
+/* Which tcgen05 kernel serves the experts above the row threshold (prefill-sized work, Section V-B's fused
+ * dequantize + tensor-core GEMM):
+ *   DYNAMO_PREFILL_PAIR (default): thread-block clusters of two CTAs; one MMA spans both SMs' tensor cores
+ *       (256 weight rows x up to 256 tokens), each CTA dequantizes its 128 rows into its own tensor memory;
+ *   DYNAMO_PREFILL_SINGLE: one CTA per SM, 256 weight rows x up to 128 tokens per work item.
+ * Both implement the same arithmetic definition.  Host-side setting; takes effect at the next forward.
+ * Errors: NULL ctx -> ERR_NULL; unknown kind -> ERR_SHAPE. */
+enum { DYNAMO_PREFILL_PAIR = 0, DYNAMO_PREFILL_SINGLE = 1 };
+dynamo_status dynamo_set_prefill_kernel(dynamo_ctx* ctx, int32_t kind);
+
 /* Measurement hook: three cudaEvent_t handles (any may be NULL) that every following forward records on
  * its stream before the gate/up FFN launch, after it, and after the down FFN launch, so that a
  * harness can time the dominant kernels in place.  Pass NULLs to switch it off. */

@@ -25,6 +25,7 @@ MAT_GATE, MAT_UP, MAT_DOWN = 0, 1, 2
 CODES_BASE, CODES_HI_POOL, CODES_HI_ACTIVE = 0, 1, 2
 SWITCH_SELECT, SWITCH_REQUANT = 0, 1
 DECODE_TENSOR, DECODE_STREAM = 0, 1
+PREFILL_PAIR, PREFILL_SINGLE = 0, 1
 
 STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_BITS", "ERR_ALIGN", "ERR_ARENA_TOO_SMALL", "ERR_INDEX_RANGE",
                 "ERR_INDEX_DUP", "ERR_NOT_CACHED", "ERR_STATE", "ERR_TOKENS", "ERR_CUDA", "ERR_TIMEOUT"]
@@ -32,7 +33,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_BITS", "ERR_ALIGN", "ERR_ARE
 EXPORTED = ["dynamo_create", "dynamo_destroy", "dynamo_arena_bytes", "dynamo_pack_experts",
             "dynamo_set_channel_switch", "dynamo_set_channel_switch_many", "dynamo_set_switch_mode",
             "dynamo_moe_forward", "dynamo_moe_forward_host", "dynamo_export_codes", "dynamo_expert_stream_bytes",
-            "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_decode_kernel", "dynamo_route_permute_static", "dynamo_kernel_launches", "dynamo_status_str"]
+            "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_decode_kernel", "dynamo_set_prefill_kernel", "dynamo_route_permute_static", "dynamo_kernel_launches", "dynamo_status_str"]
 
 
 class LayerDesc(ctypes.Structure):
@@ -77,6 +78,7 @@ def load():
         L.dynamo_set_profile_events.argtypes = [vp, vp, vp, vp]
         L.dynamo_set_tc_min_rows.argtypes = [vp, i32]
         L.dynamo_set_decode_kernel.argtypes = [vp, i32]
+        L.dynamo_set_prefill_kernel.argtypes = [vp, i32]
         L.dynamo_route_permute_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
         L.dynamo_kernel_launches.argtypes = [vp]
         L.dynamo_kernel_launches.restype = ctypes.c_int64
@@ -164,6 +166,10 @@ def dynamo_set_tc_min_rows(ctx, rows: int) -> int:
 
 def dynamo_set_decode_kernel(ctx, kind: int) -> int:
     return load().dynamo_set_decode_kernel(ctx, kind)
+
+
+def dynamo_set_prefill_kernel(ctx, kind: int) -> int:
+    return load().dynamo_set_prefill_kernel(ctx, kind)
 
 
 def dynamo_set_profile_events(ctx, e0, e1, e2) -> int:
@@ -302,6 +308,9 @@ class DynamoLayer:
 
     def set_tc_min_rows(self, rows: int):
         _check(dynamo_set_tc_min_rows(self.ctx, rows), "dynamo_set_tc_min_rows")
+
+    def set_prefill_kernel(self, kind: int):
+        _check(dynamo_set_prefill_kernel(self.ctx, kind), "dynamo_set_prefill_kernel")
 
     def set_decode_kernel(self, kind: int):
         _check(dynamo_set_decode_kernel(self.ctx, kind), "dynamo_set_decode_kernel")

@@ -25,6 +25,8 @@ cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, in
                               long long split_stride, int max_rows, int n_sms, cudaStream_t st);
 cudaError_t launch_ffn_tc(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int n_experts, int n_sms,
                           cudaStream_t st);
+cudaError_t launch_ffn_tc2(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int n_experts, int n_sms,
+                           cudaStream_t st);
 cudaError_t launch_ffn_tcd(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int ksplit, int n_experts,
                            long long split_stride, int n_sms, cudaStream_t st);
 cudaError_t launch_switch(const SwitchLayers& layers, int n_layers, int E, const int32_t* staging, int per_layer_ints,
@@ -171,7 +173,8 @@ struct dynamo_ctx {
     LayerDev host_layer;                         // host mirror of the arena header
     int switch_mode = DYNAMO_SWITCH_SELECT;
     int tc_min_rows = TC_MIN_ROWS;               // experts with more rows take the tcgen05 path
-    int decode_kernel = DYNAMO_DECODE_STREAM;     // which kernel serves forwards of up to DECODE_FOLD_TOKENS tokens
+    int decode_kernel = DYNAMO_DECODE_STREAM;
+    int prefill_kernel = DYNAMO_PREFILL_PAIR;    // which tcgen05 kernel serves experts above the row threshold    // which kernel serves forwards of up to DECODE_FOLD_TOKENS tokens
     int n_sms = 148;                             // SM count of the device the layer was packed on
     int64_t launches = 0;
     cudaEvent_t prof_ev[3] = {nullptr, nullptr, nullptr};  // optional: before gate/up, after gate/up, after down
@@ -315,6 +318,13 @@ dynamo_status dynamo_set_tc_min_rows(dynamo_ctx* ctx, int32_t rows) {
     if (rows < 0) return DYNAMO_ERR_SHAPE;
     // the streaming path handles one 32-token chunk per expert when both paths are active
     ctx->tc_min_rows = rows == 0 ? 0x7fffffff : (rows < TC_MIN_ROWS ? rows : TC_MIN_ROWS);
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_set_prefill_kernel(dynamo_ctx* ctx, int32_t kind) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    if (kind != DYNAMO_PREFILL_PAIR && kind != DYNAMO_PREFILL_SINGLE) return DYNAMO_ERR_SHAPE;
+    ctx->prefill_kernel = kind;
     return DYNAMO_OK;
 }
 
@@ -552,10 +562,13 @@ dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* ro
     if (ctx->prof_ev[0]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[0], st));
     const int max_rows = use_tc ? std::min(T, ctx->tc_min_rows) : T;  // rows one expert can have on the streaming path
     CUDA_TRY(launch_ffn_stream(L, ws, 1, ctx->host_layer.n_rb13, 1, n, split_stride, max_rows, ctx->n_sms, st));
-    if (use_tc) CUDA_TRY(launch_ffn_tc(L, ws, 1, ctx->host_layer.n_rb13, n, ctx->n_sms, st));
+    const bool pair = ctx->prefill_kernel == DYNAMO_PREFILL_PAIR;
+    if (use_tc) CUDA_TRY(pair ? launch_ffn_tc2(L, ws, 1, ctx->host_layer.n_rb13, n, ctx->n_sms, st)
+                              : launch_ffn_tc(L, ws, 1, ctx->host_layer.n_rb13, n, ctx->n_sms, st));
     if (ctx->prof_ev[1]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[1], st));
     CUDA_TRY(launch_ffn_stream(L, ws, 0, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, max_rows, ctx->n_sms, st));
-    if (use_tc) CUDA_TRY(launch_ffn_tc(L, ws, 0, ctx->host_layer.n_rb2, n, ctx->n_sms, st));
+    if (use_tc) CUDA_TRY(pair ? launch_ffn_tc2(L, ws, 0, ctx->host_layer.n_rb2, n, ctx->n_sms, st)
+                              : launch_ffn_tc(L, ws, 0, ctx->host_layer.n_rb2, n, ctx->n_sms, st));
     if (ctx->prof_ev[2]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[2], st));
     CUDA_TRY(launch_combine(ws, D.d_model, D.top_k, D.n_shared, y, y_dtype == DYNAMO_F32, split_stride, st));
     ctx->launches += use_tc ? 8 : 6;

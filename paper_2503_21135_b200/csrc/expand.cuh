@@ -98,4 +98,11 @@ __device__ __forceinline__ void expand(const Codes<BITS>& c, uint32_t (&a)[4]) {
     }
 }
 
+// In-place bit offset o of the code of (MMA step S4 of a half chunk, k pair h): see layout.cuh.
+template <int BITS>
+__host__ __device__ constexpr int code_offset(int s4, int h) {
+    const int phi = 2 * s4 + h;
+    return BITS == 2 ? (phi <= 4 ? 2 * phi : 2 * phi - 10) : BITS == 3 ? 2 * (phi & 3) : BITS == 4 ? 4 * h : 0;
+}
+
 }  // namespace dyn

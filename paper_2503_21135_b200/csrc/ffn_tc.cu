@@ -57,13 +57,6 @@ struct TcBars {
     volatile int poison;
 };
 
-// In-place bit offset o of the code of (MMA step S4 of a half chunk, k pair h): see layout.cuh.
-template <int BITS>
-__host__ __device__ constexpr int code_offset(int s4, int h) {
-    const int phi = 2 * s4 + h;
-    return BITS == 2 ? (phi <= 4 ? 2 * phi : 2 * phi - 10) : BITS == 3 ? 2 * (phi & 3) : BITS == 4 ? 4 * h : 0;
-}
-
 // Dequantize one packed block stage into the A buffer: this warp's two atoms, eight MMA steps.
 template <int BITS>
 __device__ __forceinline__ void tc_dequant_stage(const uint8_t* st, uint32_t a_lanes, int atom0, int lane, int G) {
