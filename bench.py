@@ -292,7 +292,8 @@ def run_ours(args, rank, world, device):
         achieved = gu_flops / (r["gu_ms"] / 1e3) / 1e12
         out["roofline"] = {"bound": "tensor", "achieved": achieved, "peak": tensor_peak, "unit": "TFLOP/s",
                            "frac": achieved / tensor_peak, "traffic": None, "peak_kind": peak_kind + " (sustained fp16/bf16)",
-                           "kernel": "ffn_tc_kernel<gate/up> (+ streaming kernel for experts of <= 32 rows)",
+                           "kernel": ("ffn_tc_kernel<gate/up>" if args.prefill_kernel == "single" else "ffn_tc2_kernel<gate/up>")
+                           + " (+ streaming kernel for experts of <= 32 rows)",
                            "algorithmic_flops_per_launch": gu_flops, "avg_launch_ms": r["gu_ms"],
                            "down_launch": {"achieved": gu_flops / 2 / (r["dn_ms"] / 1e3) / 1e12, "avg_launch_ms": r["dn_ms"]},
                            "whole_step_tflops": 1.5 * gu_flops / (ms_step / 1e3) / 1e12}
