@@ -29,7 +29,8 @@
 
 namespace dyn {
 
-constexpr int CONSUMER_WARPS = 8;
+constexpr int APW = 2;                 // atoms (16 weight rows) per consumer warp (1: more warps, measured slower)
+constexpr int CONSUMER_WARPS = 16 / APW;
 constexpr int FFN_THREADS = (CONSUMER_WARPS + 1) * 32;
 constexpr int SMEM_HEADER = 2048;     // barriers, poison flag, per-expert item prefix table
 constexpr int MAX_STAGES = 16;        // ring queue depth; the ring itself is byte-granular
@@ -88,7 +89,7 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
     const ExpertDev& ex = L->ex[im.e];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = lane >> 2, tid4 = lane & 3;
-    const int atom0 = warp * 2;
+    const int atom0 = warp * APW;
     const int G = L->G;
     const int K = GATEUP ? L->d : L->f;
     const int n_kc = K / KC;
@@ -103,9 +104,9 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
     const int n_ps = sig_cnt > 0 ? (L->P_pad >> 5) : 0;
     volatile int* poison = &S->poison;
 
-    float total[2][NT8][4];
+    float total[APW][NT8][4];
 #pragma unroll
-    for (int a = 0; a < 2; ++a)
+    for (int a = 0; a < APW; ++a)
 #pragma unroll
         for (int j = 0; j < NT8; ++j)
 #pragma unroll
@@ -121,9 +122,9 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
         const uint8_t* st = stages + S->off[s];
         const uint8_t* xs = st + blk_bytes;
         const uint32_t* prm = reinterpret_cast<const uint32_t*>(st + code_bytes);
-        float accg[2][NT8][4];
+        float accg[APW][NT8][4];
 #pragma unroll
-        for (int a = 0; a < 2; ++a)
+        for (int a = 0; a < APW; ++a)
 #pragma unroll
             for (int j = 0; j < NT8; ++j)
 #pragma unroll
@@ -131,9 +132,9 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
 
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
-            Codes<BITS> cd[2];
+            Codes<BITS> cd[APW];
 #pragma unroll
-            for (int a = 0; a < 2; ++a) load_codes<BITS>(cd[a], st + (atom0 + a) * atom_bytes(BITS), lane, half);
+            for (int a = 0; a < APW; ++a) load_codes<BITS>(cd[a], st + (atom0 + a) * atom_bytes(BITS), lane, half);
 
             auto step = [&](auto S4c) {
                 constexpr int S4 = decltype(S4c)::value;
@@ -147,7 +148,7 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
                     b1[j] = v.y;
                 }
 #pragma unroll
-                for (int a = 0; a < 2; ++a) {
+                for (int a = 0; a < APW; ++a) {
                     uint32_t af[4];
                     expand<BITS, S4>(cd[a], af);
 #pragma unroll
@@ -171,7 +172,7 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
                     else { xs0[j] = sa.x + sa.y; xs1[j] = sb.x + sb.y; }
                 }
 #pragma unroll
-                for (int a = 0; a < 2; ++a) {
+                for (int a = 0; a < APW; ++a) {
                     const int r0 = (atom0 + a) * 16 + gid;
                     const uint32_t p0 = prm[r0 * ngrp + g], p1 = prm[(r0 + 8) * ngrp + g];
                     const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&p0));
@@ -211,7 +212,7 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
                     b1[j] = *reinterpret_cast<const uint32_t*>(xs + (8 * j + gid) * XPOOL_ROW + (16 * ks + 2 * tid4 + 8) * 2);
                 }
 #pragma unroll
-                for (int a = 0; a < 2; ++a) {
+                for (int a = 0; a < APW; ++a) {
                     uint32_t af[4];
                     const uint32_t addr = smem_u32(st + (16 * ks + (mi >> 1) * 8 + r) * POOL_TILE_PITCH +
                                                    (16 * (atom0 + a) + (mi & 1) * 8) * 2);
@@ -231,7 +232,7 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
         // SwiGLU: rows 0..7 of an atom are gate, rows 8..15 the matching up rows.
         uint8_t* htile = htiles + (item_idx & 1) * p.htile_bytes;
 #pragma unroll
-        for (int a = 0; a < 2; ++a)
+        for (int a = 0; a < APW; ++a)
 #pragma unroll
             for (int j = 0; j < NT8; ++j)
 #pragma unroll
@@ -266,7 +267,7 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
         float* yb = p.ws.ypart + (size_t)im.split * p.split_stride;
         const int d = L->d;
 #pragma unroll
-        for (int a = 0; a < 2; ++a)
+        for (int a = 0; a < APW; ++a)
 #pragma unroll
             for (int j = 0; j < NT8; ++j)
 #pragma unroll
@@ -297,7 +298,7 @@ __device__ __forceinline__ bool consume_dispatch(const FfnParams& p, FfnSmem* S,
 }
 
 template <bool GATEUP, int MAXNT8>
-__global__ void __launch_bounds__(FFN_THREADS, MAXNT8 <= 2 ? 3 : 2) ffn_stream_kernel(const FfnParams p) {
+__global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2) ffn_stream_kernel(const FfnParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     pdl_prologue();
     if (*p.ws.status != STATUS_OK) return;  // after an expired wait nothing new starts
@@ -452,8 +453,9 @@ cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, in
                               long long split_stride, int max_rows, int n_sms, cudaStream_t st) {
     // three CTAs per SM pay off once every CTA has several items to walk; at 1-3 tokens a CTA sees one or two
     const bool small = max_rows >= 4 && max_rows <= 16;
-    const int smem_bytes = small ? 74 * 1024 : 110 * 1024;
-    const int n_ctas = (small ? 3 : 2) * n_sms;
+    const bool three = small && APW == 2;
+    const int smem_bytes = three ? 74 * 1024 : 110 * 1024;
+    const int n_ctas = (three ? 3 : 2) * n_sms;
     FfnParams p;
     p.L = L;
     p.ws = ws;

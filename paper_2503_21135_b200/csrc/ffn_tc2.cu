@@ -87,7 +87,7 @@ __device__ __forceinline__ T2Item t2_decode_item(const T2Params& p, const int* p
     const int local = g - prefix[cursor];
     const int cnt = p.ws.counts[e];
     const int n_tt = (cnt + T2_N - 1) / T2_N;
-    const int tt = local % n_tt;
+    const int tt = local % n_tt;  // tiles of one weight block are neighbours: concurrent clusters share its L2 lines
     T2Item it;
     it.rb = local / n_tt;
     it.n_valid = min(T2_N, cnt - tt * T2_N);
