@@ -245,6 +245,23 @@ def run_ours(args, rank, world, device):
         res["gu_ms"], res["dn_ms"] = kernel_times(layers, step, args.steps)
         results[Tcur] = res
 
+    router = None
+    if args.router:
+        # the same step with the router GEMM + top-k fused in front (scores from synthetic router weights, so the
+        # routing differs from the logits-input run above: compare times at token counts where every expert is active)
+        wr = [wl.router_weights(cfg, l) for l in range(n_layers)]
+        wrd = [(w.to(device), b.to(device)) for w, b in wr]
+        xs = [wl.activations(cfg, T, l, step=0).to(device) for l in range(n_layers)]
+
+        def step_router(i):
+            l = i % n_layers
+            layers[l].forward_router(xs[l], wrd[l][0], wrd[l][1], binding.F32)
+
+        for i in range(max(args.warmup, 3)):
+            step_router(i)
+        ms_r = time_steps(step_router, args.steps, barrier)
+        router = {"ms_per_step_with_router_gemm": ms_r / args.steps, "tokens_per_s": world * T / (ms_r / args.steps / 1e3)}
+
     # end-to-end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     xh = [wl.activations(cfg, T, l, step=0).pin_memory() for l in range(n_layers)]
     lh = [wl.router_logits(cfg, T, l, step=0).pin_memory() for l in range(n_layers)]
@@ -309,6 +326,8 @@ def run_ours(args, rank, world, device):
                        "down_launch": {"achieved": r["dn_bytes"] / (r["dn_ms"] / 1e3) / 1e9, "avg_launch_ms": r["dn_ms"]},
                        "whole_step": {"achieved": r["bytes_per_step"] / (ms_step / 1e3) / 1e9,
                                       "frac": r["bytes_per_step"] / (ms_step / 1e3) / 1e9 / hbm_peak}}
+    if router is not None:
+        out["router"] = router
     out["extra"] = {str(t): {"tokens_per_s": world * t / (v["ms_per_step"] / 1e3), "ms_per_step": v["ms_per_step"],
                              "gateup_ms": v["gu_ms"], "down_ms": v["dn_ms"],
                              "step_gbs": v["bytes_per_step"] / (v["ms_per_step"] / 1e3) / 1e9,
@@ -449,6 +468,8 @@ def main():
                     help="tcgen05 kernel for experts above the row threshold (default: the library's, pair)")
     ap.add_argument("--decode-kernel", default=None, choices=["tensor", "stream"],
                     help="kernel for batches of up to 64 tokens (default: the library's, stream)")
+    ap.add_argument("--router", action="store_true",
+                    help="also time the forward with the router GEMM + top-k fused in front")
     ap.add_argument("--sweep", action="store_true", help="also time the workload's other token counts")
     ap.add_argument("--cpu-tokens", type=int, default=16, help="tokens in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -148,6 +148,21 @@ dynamo_status dynamo_set_switch_mode(dynamo_ctx* ctx, int32_t mode);
 dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* router_logits, int32_t T,
                                  void* y, int32_t y_dtype, const dynamo_debug_out* dbg, void* stream);
 
+/* The same forward with the router's scoring fused in front (Section II-A: the gating network scores every
+ * expert for a token, the K best are taken):
+ *   logits[t][e] = sum_c x[t][c] * w_router[e][c] + router_bias[e]      (bf16 inputs, fp32 accumulation in a
+ *   fixed order: deterministic), then top-k and softmax exactly as above, in the same kernel.
+ *   w_router    : dev bf16 [E, d], 16-byte aligned (as x must be)
+ *   router_bias : dev fp32 [E] or NULL
+ *   logits_out  : dev fp32 [T, E] or NULL: where to store the computed scores (parity tests)
+ * Because the scores are rounded in fp32, two experts whose exact scores differ by less than the accumulation
+ * error may be ordered differently than by exact arithmetic; given the scores written to logits_out the
+ * selection is exactly the rule above.  Errors as dynamo_moe_forward; NULL w_router -> ERR_NULL; misaligned
+ * x or w_router -> ERR_ALIGN. */
+dynamo_status dynamo_moe_forward_router(dynamo_ctx* ctx, const void* x, const void* w_router,
+                                        const float* router_bias, int32_t T, void* y, int32_t y_dtype,
+                                        float* logits_out, const dynamo_debug_out* dbg, void* stream);
+
 /* Same forward with HOST buffers: copies x and the logits to the device, runs the forward,
  * copies y back and synchronises the stream before returning.  Pinned host memory makes the
  * copies asynchronous with respect to other streams; pageable memory works too. */

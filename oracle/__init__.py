@@ -62,6 +62,8 @@ def lib():
         L.orc_pack_rows.argtypes = [u8p, i64, i64, ci, u32p]
         L.orc_unpack_rows.restype = None
         L.orc_unpack_rows.argtypes = [u32p, i64, i64, ci, u8p]
+        L.orc_router_scores.restype = None
+        L.orc_router_scores.argtypes = [u16p, u16p, f32p, i64, i64, ci, f64p]
         L.orc_route.restype = None
         L.orc_route.argtypes = [f32p, i64, ci, ci, ci, i32p, f64p]
         L.orc_permute.restype = None
@@ -152,6 +154,20 @@ def unpack_rows(words: np.ndarray, K: int, bits: int) -> np.ndarray:
 
 
 # ---- C3 / C4 -------------------------------------------------------------------------------
+
+def router_scores(x_u16: np.ndarray, w_u16: np.ndarray, bias: Optional[np.ndarray] = None) -> np.ndarray:
+    """Router scores float64 [T, E] = x . w_r^T + bias from bf16 bit patterns (Section II-A)."""
+    x_u16 = np.ascontiguousarray(x_u16, dtype=np.uint16)
+    w_u16 = np.ascontiguousarray(w_u16, dtype=np.uint16)
+    T, d = x_u16.shape
+    E = w_u16.shape[0]
+    assert w_u16.shape[1] == d
+    b = None if bias is None else np.ascontiguousarray(bias, dtype=np.float32)
+    out = np.empty((T, E), dtype=np.float64)
+    lib().orc_router_scores(_p(x_u16, ctypes.c_uint16), _p(w_u16, ctypes.c_uint16), _p(b, ctypes.c_float), T, d, E,
+                            _p(out, ctypes.c_double))
+    return out
+
 
 def route(logits: np.ndarray, k: int, renormalize: bool = True):
     """Top-k routing.  logits fp32 [T,E] -> (idx int32 [T,k], w float64 [T,k])."""

@@ -151,6 +151,19 @@ void orc_unpack_rows(const uint32_t* in, int64_t N, int64_t K, int bits, uint8_t
         }
 }
 
+/* ---- router scores (Section II-A: the gating network scores every expert for a token) -------
+ * scores[t][e] = sum_c x[t][c] * w_r[e][c] + bias[e]; x and w_r are bf16 bit patterns, every product and
+ * the sum in double (a product of two bf16 values is exact in double; the sum of d of them rounds at 2^-53). */
+void orc_router_scores(const uint16_t* x, const uint16_t* w_r, const float* bias, int64_t T, int64_t d, int E,
+                       double* scores) {
+    for (int64_t t = 0; t < T; ++t)
+        for (int e = 0; e < E; ++e) {
+            double acc = 0.0;
+            for (int64_t c = 0; c < d; ++c) acc += orc_bf16_to_f64(x[t * d + c]) * orc_bf16_to_f64(w_r[(int64_t)e * d + c]);
+            scores[t * E + e] = acc + (bias ? (double)bias[e] : 0.0);
+        }
+}
+
 /* ---- C3: Top-K routing (Section II-A: a fixed number of experts per token) ------------
  * idx[t, :] = the k experts with the largest logits, descending, ties -> lower index.
  * p = softmax(logits[t, :]) in double over all E; w = p[idx] (divided by their sum if renorm). */

@@ -32,7 +32,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_BITS", "ERR_ALIGN", "ERR_ARE
 
 EXPORTED = ["dynamo_create", "dynamo_destroy", "dynamo_arena_bytes", "dynamo_pack_experts",
             "dynamo_set_channel_switch", "dynamo_set_channel_switch_many", "dynamo_set_switch_mode",
-            "dynamo_moe_forward", "dynamo_moe_forward_host", "dynamo_export_codes", "dynamo_expert_stream_bytes",
+            "dynamo_moe_forward", "dynamo_moe_forward_router", "dynamo_moe_forward_host", "dynamo_export_codes", "dynamo_expert_stream_bytes",
             "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_decode_kernel", "dynamo_set_prefill_kernel", "dynamo_route_permute_static", "dynamo_kernel_launches", "dynamo_status_str"]
 
 
@@ -72,6 +72,7 @@ def load():
         L.dynamo_set_switch_mode.argtypes = [vp, i32]
         L.dynamo_moe_forward.argtypes = [vp, vp, vp, i32, vp, i32, ctypes.POINTER(DebugOut), vp]
         L.dynamo_moe_forward_host.argtypes = [vp, vp, vp, i32, vp, i32, vp]
+        L.dynamo_moe_forward_router.argtypes = [vp, vp, vp, vp, i32, vp, i32, vp, ctypes.POINTER(DebugOut), vp]
         L.dynamo_export_codes.argtypes = [vp, i32, i32, vp, vp, vp, i32, vp]
         L.dynamo_expert_stream_bytes.argtypes = [vp, i32, ctypes.POINTER(sz)]
         L.dynamo_poll_status.argtypes = [vp, vp]
@@ -140,6 +141,11 @@ def dynamo_set_switch_mode(ctx, mode: int) -> int:
 def dynamo_moe_forward(ctx, x, logits, T, y, y_dtype, dbg: Optional[DebugOut], stream) -> int:
     return load().dynamo_moe_forward(ctx, x, logits, T, y, y_dtype, ctypes.byref(dbg) if dbg is not None else None,
                                      stream)
+
+
+def dynamo_moe_forward_router(ctx, x, w_router, bias, T, y, y_dtype, logits_out, dbg: Optional[DebugOut], stream) -> int:
+    return load().dynamo_moe_forward_router(ctx, x, w_router, bias, T, y, y_dtype, logits_out,
+                                            ctypes.byref(dbg) if dbg is not None else None, stream)
 
 
 def dynamo_moe_forward_host(ctx, x_host, logits_host, T, y_host, y_dtype, stream) -> int:
@@ -283,6 +289,32 @@ class DynamoLayer:
         st = dynamo_moe_forward(self.ctx, x.data_ptr(), logits.data_ptr(), T, y.data_ptr(), y_dtype, dbg, _stream())
         _check(st, "dynamo_moe_forward")
         return (y, outs) if debug else y
+
+    def forward_router(self, x: torch.Tensor, w_router: torch.Tensor, bias: Optional[torch.Tensor] = None, y_dtype=F32,
+                       want_logits=False, debug=False):
+        """Forward with the router GEMM + top-k fused in front; returns y (, logits) (, debug outputs)."""
+        T = x.shape[0]
+        E, k = self.desc.n_experts, self.desc.top_k
+        assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
+        assert w_router.is_cuda and w_router.dtype == torch.bfloat16 and w_router.is_contiguous()
+        assert tuple(w_router.shape) == (E, self.desc.d_model)
+        assert bias is None or (bias.is_cuda and bias.dtype == torch.float32 and bias.numel() == E)
+        y = torch.empty((T, self.desc.d_model), dtype=torch.float32 if y_dtype == F32 else torch.bfloat16, device=x.device)
+        lg = torch.empty((T, E), dtype=torch.float32, device=x.device) if want_logits else None
+        dbg, outs = None, None
+        if debug:
+            outs = {"idx": torch.empty((T, k), dtype=torch.int32, device=x.device),
+                    "w": torch.empty((T, k), dtype=torch.float32, device=x.device),
+                    "offsets": torch.empty((E + 1,), dtype=torch.int32, device=x.device),
+                    "perm": torch.empty((T * k,), dtype=torch.int32, device=x.device)}
+            dbg = DebugOut(outs["idx"].data_ptr(), outs["w"].data_ptr(), outs["offsets"].data_ptr(),
+                           outs["perm"].data_ptr())
+        st = dynamo_moe_forward_router(self.ctx, x.data_ptr(), w_router.data_ptr(),
+                                       bias.data_ptr() if bias is not None else None, T, y.data_ptr(), y_dtype,
+                                       lg.data_ptr() if lg is not None else None, dbg, _stream())
+        _check(st, "dynamo_moe_forward_router")
+        res = (y,) + ((lg,) if want_logits else ()) + ((outs,) if debug else ())
+        return res if len(res) > 1 else y
 
     def forward_host(self, x_host: torch.Tensor, logits_host: torch.Tensor, y_host: torch.Tensor, y_dtype=F32):
         T = x_host.shape[0]

@@ -17,6 +17,8 @@ cudaError_t launch_export(const LayerDev* L, int e, int mat, int which, long lon
                           uint16_t* zr, cudaStream_t st);
 cudaError_t launch_route(const float* logits, int T, int E, int k, int renorm, int32_t* idx, float* w,
                          cudaStream_t st);
+cudaError_t launch_route_gemm(const void* x, const void* w_router, const float* bias, int T, int d, int E, int k,
+                              int renorm, float* logits_out, int32_t* idx, float* w, cudaStream_t st);
 cudaError_t launch_scan(const WsDev& ws, int E, int Es, int k, cudaStream_t st);
 cudaError_t launch_gather(const LayerDev* L, const WsDev& ws, const void* x, cudaStream_t st);
 cudaError_t launch_combine(const WsDev& ws, int d, int k, int Es, void* y, int y_f32, long long split_stride,
@@ -530,21 +532,29 @@ static dynamo_status forward_debug_copies(const dynamo_ctx* ctx, const WsDev& ws
     return DYNAMO_OK;
 }
 
-dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* router_logits, int32_t T, void* y,
-                                 int32_t y_dtype, const dynamo_debug_out* dbg, void* stream) {
+// The forward from either given router logits or the router's weights (then the scores are computed by the
+// fused GEMM + top-k kernel, and written to logits_out if that is not NULL).
+static dynamo_status forward_impl(dynamo_ctx* ctx, const void* x, const float* router_logits, const void* w_router,
+                                  const float* router_bias, float* logits_out, int32_t T, void* y, int32_t y_dtype,
+                                  const dynamo_debug_out* dbg, void* stream) {
     if (!ctx) return DYNAMO_ERR_NULL;
     if (!ctx->packed) return DYNAMO_ERR_STATE;
     const dynamo_layer_desc& D = ctx->D;
     if (T < 0 || T > D.max_tokens) return DYNAMO_ERR_TOKENS;
     if (y_dtype != DYNAMO_BF16 && y_dtype != DYNAMO_F32) return DYNAMO_ERR_SHAPE;
     if (T == 0) return DYNAMO_OK;
-    if (!x || !router_logits || !y) return DYNAMO_ERR_NULL;
+    if (!x || (!router_logits && !w_router) || !y) return DYNAMO_ERR_NULL;
+    if (w_router && (((uintptr_t)w_router | (uintptr_t)x) & 15)) return DYNAMO_ERR_ALIGN;  // 16-byte vector loads
     cudaStream_t st = (cudaStream_t)stream;
     const LayerDev* L = (const LayerDev*)ctx->arena;
     WsDev ws = make_ws(ctx, T);
     const int n = D.n_experts + D.n_shared;
 
-    CUDA_TRY(launch_route(router_logits, T, D.n_experts, D.top_k, D.renormalize, ws.topk_idx, ws.topk_w, st));
+    if (w_router)
+        CUDA_TRY(launch_route_gemm(x, w_router, router_bias, T, D.d_model, D.n_experts, D.top_k, D.renormalize, logits_out,
+                                   ws.topk_idx, ws.topk_w, st));
+    else
+        CUDA_TRY(launch_route(router_logits, T, D.n_experts, D.top_k, D.renormalize, ws.topk_idx, ws.topk_w, st));
     CUDA_TRY(launch_scan(ws, D.n_experts, D.n_shared, D.top_k, st));
     CUDA_TRY(launch_gather(L, ws, x, st));
     const bool use_tc = ws.tc_min != 0x7fffffff;                  // experts above 32 rows take the tcgen05 path
@@ -573,6 +583,19 @@ dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* ro
     CUDA_TRY(launch_combine(ws, D.d_model, D.top_k, D.n_shared, y, y_dtype == DYNAMO_F32, split_stride, st));
     ctx->launches += use_tc ? 8 : 6;
     return forward_debug_copies(ctx, ws, T, dbg, st);
+}
+
+dynamo_status dynamo_moe_forward(dynamo_ctx* ctx, const void* x, const float* router_logits, int32_t T, void* y,
+                                 int32_t y_dtype, const dynamo_debug_out* dbg, void* stream) {
+    if (ctx && ctx->packed && T > 0 && T <= ctx->D.max_tokens && !router_logits) return DYNAMO_ERR_NULL;
+    return forward_impl(ctx, x, router_logits, nullptr, nullptr, nullptr, T, y, y_dtype, dbg, stream);
+}
+
+dynamo_status dynamo_moe_forward_router(dynamo_ctx* ctx, const void* x, const void* w_router, const float* router_bias,
+                                        int32_t T, void* y, int32_t y_dtype, float* logits_out,
+                                        const dynamo_debug_out* dbg, void* stream) {
+    if (ctx && ctx->packed && T > 0 && T <= ctx->D.max_tokens && !w_router) return DYNAMO_ERR_NULL;
+    return forward_impl(ctx, x, nullptr, w_router, router_bias, logits_out, T, y, y_dtype, dbg, stream);
 }
 
 dynamo_status dynamo_moe_forward_host(dynamo_ctx* ctx, const void* x_host, const float* logits_host, int32_t T,

@@ -14,21 +14,14 @@
 
 namespace dyn {
 
-// One warp per token.  E <= 256: lane l holds logits l, l+32, ...
-__global__ void __launch_bounds__(256) route_kernel(const float* __restrict__ logits, int T, int E, int k, int renorm,
-                                                    int32_t* __restrict__ topk_idx, float* __restrict__ topk_w) {
-    pdl_prologue();
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-    if (warp >= T) return;
-    const float* l = logits + (long long)warp * E;
-    float v[8];
+// Top-k of one token's logits held across a warp (lane l holds logits l, l+32, ...; E <= 256): k largest raw
+// logits, descending, ties -> lower expert index; weights = softmax over all E restricted to the chosen,
+// rescaled to sum 1 if `renorm`.
+__device__ __forceinline__ void topk_softmax_store(float (&v)[8], int lane, int E, int k, int renorm, long long token,
+                                                   int32_t* __restrict__ topk_idx, float* __restrict__ topk_w) {
     float mx = -INFINITY;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const int e = lane + 32 * i;
-        v[i] = (e < E) ? l[e] : -INFINITY;
-        mx = fmaxf(mx, v[i]);
-    }
+    for (int i = 0; i < 8; ++i) mx = fmaxf(mx, v[i]);
 #pragma unroll
     for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     float den = 0.f;
@@ -66,10 +59,92 @@ __global__ void __launch_bounds__(256) route_kernel(const float* __restrict__ lo
     }
     if (lane == 0) {
         for (int j = 0; j < k; ++j) {
-            topk_idx[(long long)warp * k + j] = isel[j];
-            topk_w[(long long)warp * k + j] = renorm ? wsel[j] / wsum : wsel[j];
+            topk_idx[token * k + j] = isel[j];
+            topk_w[token * k + j] = renorm ? wsel[j] / wsum : wsel[j];
         }
     }
+}
+
+// One warp per token.
+__global__ void __launch_bounds__(256) route_kernel(const float* __restrict__ logits, int T, int E, int k, int renorm,
+                                                    int32_t* __restrict__ topk_idx, float* __restrict__ topk_w) {
+    pdl_prologue();
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= T) return;
+    const float* l = logits + (long long)warp * E;
+    float v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int e = lane + 32 * i;
+        v[i] = (e < E) ? l[e] : -INFINITY;
+    }
+    topk_softmax_store(v, lane, E, k, renorm, warp, topk_idx, topk_w);
+}
+
+// Router GEMM fused with the top-k (Section II-A: the gate scores every expert, the K best are taken):
+// logits[t][e] = sum_c x[t][c] * W_r[e][c] (+ bias[e]), bf16 inputs, fp32 accumulate.  One CTA of eight warps
+// per token: warp w, lane l take the input indices 8*l + 256*(w + 8*i) ..+7; every warp reduces its partial
+// sums over its lanes by a fixed butterfly, the eight partials are added in warp order, so the sum order
+// (hence the fp32 result) is deterministic.  The products of two bf16 values are exact in fp32; only the
+// additions round.  Warp 0 then selects the top-k exactly as route_kernel does.
+__global__ void __launch_bounds__(256) route_gemm_kernel(const __nv_bfloat16* __restrict__ x,
+                                                         const __nv_bfloat16* __restrict__ w_router,
+                                                         const float* __restrict__ bias, int T, int d, int E, int k,
+                                                         int renorm, float* __restrict__ logits_out,
+                                                         int32_t* __restrict__ topk_idx, float* __restrict__ topk_w) {
+    __shared__ float part[8][MAX_EXPERTS];
+    pdl_prologue();
+    const int token = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const __nv_bfloat16* xr = x + (long long)token * d;
+    for (int e0 = 0; e0 < E; e0 += 8) {  // eight experts at a time
+        float acc[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+        for (int c = 8 * lane + 256 * warp; c < d; c += 2048) {
+            const uint4 xv = *reinterpret_cast<const uint4*>(xr + c);
+            const __nv_bfloat162* xp = reinterpret_cast<const __nv_bfloat162*>(&xv);
+            float xf[8];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                xf[2 * u] = __low2float(xp[u]);
+                xf[2 * u + 1] = __high2float(xp[u]);
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (e0 + j < E) {
+                    const uint4 wv = *reinterpret_cast<const uint4*>(w_router + (long long)(e0 + j) * d + c);
+                    const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        acc[j] = fmaf(xf[2 * u], __low2float(wp[u]), acc[j]);
+                        acc[j] = fmaf(xf[2 * u + 1], __high2float(wp[u]), acc[j]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+#pragma unroll
+            for (int o = 16; o; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+            if (lane == 0 && e0 + j < E) part[warp][e0 + j] = acc[j];
+        }
+    }
+    __syncthreads();
+    if (warp != 0) return;
+    float v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int e = lane + 32 * i;
+        v[i] = -INFINITY;
+        if (e < E) {
+            float sum = part[0][e];
+#pragma unroll
+            for (int w = 1; w < 8; ++w) sum += part[w][e];
+            v[i] = sum + (bias ? bias[e] : 0.f);
+            if (logits_out) logits_out[(long long)token * E + e] = v[i];
+        }
+    }
+    topk_softmax_store(v, lane, E, k, renorm, token, topk_idx, topk_w);
 }
 
 // Single CTA of 32 warps.  The pair array (pair i = t*k + j, ascending in t) is cut into 32 contiguous
@@ -316,6 +391,11 @@ __global__ void __launch_bounds__(256) combine_kernel(WsDev ws, int d, int k, in
 cudaError_t launch_route(const float* logits, int T, int E, int k, int renorm, int32_t* idx, float* w,
                          cudaStream_t st) {
     return launch_pdl(route_kernel, dim3((unsigned)((T + 7) / 8)), dim3(256), 0, st, logits, T, E, k, renorm, idx, w);
+}
+cudaError_t launch_route_gemm(const void* x, const void* w_router, const float* bias, int T, int d, int E, int k,
+                              int renorm, float* logits_out, int32_t* idx, float* w, cudaStream_t st) {
+    return launch_pdl(route_gemm_kernel, dim3((unsigned)T), dim3(256), 0, st, (const __nv_bfloat16*)x,
+                      (const __nv_bfloat16*)w_router, bias, T, d, E, k, renorm, logits_out, idx, w);
 }
 cudaError_t launch_scan(const WsDev& ws, int E, int Es, int k, cudaStream_t st) {
     const int batches = (ws.T * k + 31) / 32;  // one warp per segment of whole 32-pair batches

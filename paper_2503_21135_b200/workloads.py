@@ -36,7 +36,7 @@ import torch
 BASE_SEED = 250321135
 
 # tensor ids of the per-stream seeds
-_T_X, _T_LOGITS, _T_OUTLIER, _T_POOL, _T_SIG, _T_BITS, _T_SWITCH = 0, 1, 2, 3, 4, 5, 6
+_T_X, _T_LOGITS, _T_OUTLIER, _T_POOL, _T_SIG, _T_BITS, _T_SWITCH, _T_ROUTER = 0, 1, 2, 3, 4, 5, 6, 7
 _T_WGATE, _T_WUP, _T_WDOWN = 10, 11, 12
 
 
@@ -173,6 +173,14 @@ def router_logits(cfg: MoEConfig, T: int, layer: int = 0, step: int = 0) -> torc
     a = _rng(cfg, layer, _T_LOGITS, step).standard_normal(size=(T, cfg.n_experts), dtype=np.float32)
     a = a.astype(np.float64) + popularity_bias(cfg)[None, :]
     return torch.from_numpy(a.astype(np.float32))
+
+
+def router_weights(cfg: MoEConfig, layer: int = 0):
+    """Router weight bf16 [E, d] ~ N(0, 1/d) (unit-variance scores for unit-variance inputs) and bias fp32 [E] =
+    the config's popularity bias: inputs of the fused router GEMM."""
+    w = _rng(cfg, layer, _T_ROUTER, 0).standard_normal(size=(cfg.n_experts, cfg.d_model), dtype=np.float32)
+    w *= np.float32(1.0 / np.sqrt(cfg.d_model))
+    return torch.from_numpy(w).to(torch.bfloat16), torch.from_numpy(popularity_bias(cfg).astype(np.float32))
 
 
 def cache_pool(cfg: MoEConfig, layer: int = 0) -> np.ndarray:

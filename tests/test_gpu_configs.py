@@ -73,6 +73,20 @@ def test_finegrained_config_with_shared_experts():
     counts = np.bincount(idx.ravel(), minlength=64)
     assert counts.min() <= 8 and counts.max() >= 1000                     # from decode-like to prefill-like experts
     _check_forward(cfg, gpu, ora, 37, 37, step=2)
+    # router GEMM + top-k fused in front (E = 64: two 32-expert register groups, k = 6, shared experts behind)
+    w_r, bias = wl.router_weights(cfg)
+    x = wl.activations(cfg, 300, 0, 5)
+    y, lg, dbg = gpu.forward_router(x.cuda(), w_r.cuda(), bias.cuda(), binding.F32, want_logits=True, debug=True)
+    torch.cuda.synchronize()
+    assert gpu.poll_status() == 0
+    lg = lg.cpu().numpy()
+    ref_scores = oracle.router_scores(oracle.as_u16(x), oracle.as_u16(w_r), bias.numpy())
+    bound = 2.0 * (cfg.d_model // 256 + 12) * 2.0 ** -24 * (np.abs(x.double().numpy()) @ np.abs(w_r.double().numpy()).T)
+    assert np.all(np.abs(lg.astype(np.float64) - ref_scores) <= bound + 1e-7)
+    idx_r, w_rt = oracle.route(lg, cfg.top_k)
+    assert np.array_equal(dbg["idx"].cpu().numpy(), idx_r)
+    assert np.max(np.abs(dbg["w"].cpu().numpy().astype(np.float64) - w_rt)) <= 1e-6
+    assert torch.equal(gpu.forward(x.cuda(), torch.from_numpy(lg).cuda(), binding.F32), y)
 
 
 def test_switch_stress_stack():

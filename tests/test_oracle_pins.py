@@ -363,3 +363,31 @@ def test_significant_channels_reduce_error_on_outliers():
     e0 = h_err()
     layer.set_channel_switch([np.array([3])])
     assert h_err() < e0
+
+
+# ---- router scores (Section II-A gating network; a "next" row of the scope table) --------------
+
+def test_router_scores_match_library_matmul_and_closed_forms():
+    rng = np.random.default_rng(77)
+    T, d, E = 9, 512, 8
+    x = bf16_bits(rng.standard_normal((T, d)))
+    w = bf16_bits(rng.standard_normal((E, d)) / np.sqrt(d))
+    b = rng.standard_normal(E).astype(np.float32)
+    xv = torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).to(torch.float64).numpy()
+    wv = torch.from_numpy(w.view(np.int16)).view(torch.bfloat16).to(torch.float64).numpy()
+    s = oracle.router_scores(x, w, b)
+    ref = xv @ wv.T + b.astype(np.float64)                       # library routine, float64
+    assert np.max(np.abs(s - ref)) <= 1e-12 * np.max(np.abs(ref))
+    assert np.array_equal(oracle.router_scores(x, w, None), s - b.astype(np.float64)[None, :]) or \
+        np.max(np.abs(oracle.router_scores(x, w, None) - (s - b.astype(np.float64)[None, :]))) <= 1e-14
+    # one-hot rows pick single input channels exactly; zero weights leave the bias
+    onehot = np.zeros((E, d))
+    cols = rng.permutation(d)[:E]
+    onehot[np.arange(E), cols] = 1.0
+    assert np.array_equal(oracle.router_scores(x, bf16_bits(onehot), None), xv[:, cols])
+    assert np.array_equal(oracle.router_scores(x, bf16_bits(np.zeros((E, d))), b), np.tile(b.astype(np.float64), (T, 1)))
+    # a transposed operand or a dropped bias would fail this hand-worked case: x = (1, 2, -3, 0.5),
+    # w0 = (1, 0, 0, 0), w1 = (0.5, 0.5, 0.5, 0.5), bias = (0, 1)  ->  (1, 0.25 + 1)
+    xs = bf16_bits(np.array([[1.0, 2.0, -3.0, 0.5]]))
+    ws = bf16_bits(np.array([[1.0, 0.0, 0.0, 0.0], [0.5, 0.5, 0.5, 0.5]]))
+    assert oracle.router_scores(xs, ws, np.array([0.0, 1.0], np.float32)).tolist() == [[1.0, 1.25]]
