@@ -46,6 +46,7 @@ struct FfnParams {
     int htile_bytes;         // bytes of one h tile behind the ring
     int n_rb;                // 256-row weight blocks of the matrix
     int n_experts;
+    int32_t* work_ctr;       // device counter of this launch's work queue (zeroed by the scan kernel)
 };
 
 struct Item {
@@ -56,6 +57,7 @@ struct FfnSmem {
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], done;
     int off[MAX_STAGES];    // ring offset of the stage in queue slot q (written by the producer before it arrives)
     int size[MAX_STAGES];   // bytes the stage holds in the ring (producer only)
+    int first_item[MAX_STAGES];  // item index if the stage opens an item, -2 if not, -1: no more items
     volatile int poison;
     int n_items;
     int prefix[MAX_EXPERTS + 1];  // items before expert order[y]
@@ -359,7 +361,34 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
         };
         const int K = GATEUP ? L->d : L->f;
         const int n_kc = K / KC;
-        for (int g = blockIdx.x; g < n_items && ok; g += gridDim.x) {
+        // Work queue: items are numbered heaviest bit-width first and handed out one at a time (an atomic counter),
+        // so a CTA that drew a light item comes back sooner: with one to three items per CTA and items that differ
+        // fourfold in bytes, a static deal leaves the CTAs with the 8-bit items far behind the rest.
+        bool first_draw = true;
+        const bool all_static = n_items <= (int)gridDim.x;  // at most one item per CTA
+        while (ok) {
+            // the first item of every CTA is dealt statically (CTA j takes item j: one per SM before any SM gets a
+            // second one, which matters when there are fewer items than CTAs), the rest come from the counter
+            int g = blockIdx.x;
+            if (!first_draw) {
+                if (all_static) break;  // every item was dealt statically: the consumers know, nothing to signal
+                if (lane == 0) g = gridDim.x + atomicAdd(p.work_ctr, 1);
+                g = __shfl_sync(0xffffffffu, g, 0);
+            } else if (all_static && g >= n_items) {
+                break;
+            }
+            first_draw = false;
+            if (g >= n_items) {  // tell the consumers: an empty stage marked -1
+                int off = 0;
+                if (lane == 0) off = acquire(128);
+                off = __shfl_sync(0xffffffffu, off, 0);
+                if (off >= 0 && lane == 0) {
+                    S->first_item[it % NS] = -1;
+                    mbar_arrive(&S->full[it % NS]);
+                }
+                break;
+            }
+            bool first = true;
             const Item im = decode_item(p, S, g, y);
             const ExpertDev& ex = L->ex[im.e];
             const int blk_bytes = ex.blk_bytes;
@@ -381,10 +410,12 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
                 uint8_t* st = stages + off;
                 if (lane == 0) {
                     // two copies per stage: the packed block and the (chunk-major, hence contiguous) activation slice
+                    S->first_item[s] = first ? g : -2;
                     mbar_arrive_expect_tx(&S->full[s], (uint32_t)(blk_bytes + im.nvalid * XROW));
                     bulk_g2s(st, wbase + (size_t)kc * blk_bytes, (uint32_t)blk_bytes, &S->full[s]);
                     bulk_g2s(st + blk_bytes, xbuf + act_off(kc, im.row0, p.ws.Rcap), (uint32_t)(im.nvalid * XROW), &S->full[s]);
                 }
+                first = false;
                 __syncwarp();
             }
             if constexpr (GATEUP) {
@@ -399,6 +430,7 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
                     if (!ok) break;
                     uint8_t* st = stages + off;
                     if (lane == 0) {
+                        S->first_item[s] = -2;
                         mbar_arrive_expect_tx(&S->full[s], (uint32_t)(POOL_GROUP * POOL_TILE_PITCH + im.nvalid * XPOOL_ROW));
                         bulk_g2s(st, reinterpret_cast<const uint8_t*>(ex.pool_hi) + pool_tile_off(im.rb, ps * POOL_GROUP, L->P_pad),
                                  POOL_GROUP * POOL_TILE_PITCH, &S->full[s]);
@@ -422,7 +454,17 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
     // ---------------- consumer warps ----------------
     int stage_it = 0, y = 0, item_idx = 0;
     (void)G;
-    for (int g = blockIdx.x; g < n_items; g += gridDim.x, ++item_idx) {
+    const bool all_static = n_items <= (int)gridDim.x;
+    for (;; ++item_idx) {
+        if (all_static && (item_idx > 0 || (int)blockIdx.x >= n_items)) return;
+        // the next stage opens the next item (or says there is none): its index rides with the stage
+        int g = blockIdx.x;  // the first item is dealt statically: decode it while its first stage is in flight
+        if (item_idx > 0) {
+            const int s0 = stage_it % NS;
+            if (!mbar_wait_bounded(&S->full[s0], (stage_it / NS) & 1, poison, p.ws.status)) return;
+            g = S->first_item[s0];
+        }
+        if (g < 0 || g >= n_items) return;
         const Item im = decode_item(p, S, g, y);
         bool ok;
         switch (L->ex[im.e].bits) {
@@ -467,6 +509,7 @@ cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, in
     p.ring_bytes = (smem_bytes - SMEM_HEADER - (gateup ? 2 * p.htile_bytes : 0)) & ~127;
     p.n_rb = n_rb;
     p.n_experts = n_experts;
+    p.work_ctr = ws.status + (gateup ? 4 : 5);
     if (small && max_rows <= 8) return gateup ? launch_one<true, 1>(p, n_ctas, st) : launch_one<false, 1>(p, n_ctas, st);
     if (small) return gateup ? launch_one<true, 2>(p, n_ctas, st) : launch_one<false, 2>(p, n_ctas, st);
     return gateup ? launch_one<true, 4>(p, n_ctas, st) : launch_one<false, 4>(p, n_ctas, st);

@@ -164,6 +164,8 @@ __global__ void __launch_bounds__(1024) scan_kernel(WsDev ws, int E, int Es, int
     const int T = ws.T, n_pairs = T * k;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
     const int kk = k + Es;
+    // work-queue counters of this forward's FFN launches (callers that only route pass no status block)
+    if (ws.status && threadIdx.x < 4) ws.status[4 + threadIdx.x] = 0;
     const int per_warp = ((n_pairs + 31) / 32 + nwarps - 1) / nwarps * 32;  // whole 32-pair batches per segment
     const int seg_lo = min(n_pairs, warp * per_warp), seg_hi = min(n_pairs, seg_lo + per_warp);
     const unsigned lt = (1u << lane) - 1;
