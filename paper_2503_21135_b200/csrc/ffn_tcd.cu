@@ -37,7 +37,7 @@ namespace dyn {
 
 constexpr int TD_EXP_WARPS = 8;                          // code expansion -> tensor memory, two atoms each
 constexpr int TD_FOLD_WARPS = 8;                         // accumulator groups -> fp32 totals, epilogue
-constexpr int TD_DEQ_WARPS = TD_EXP_WARPS + TD_FOLD_WARPS;
+
 // Warp roles.  The producer and the MMA issuers take the LOWEST warp ids: they issue few instructions but every
 // one is on the critical path, and the schedulers favour older (lower) warps.
 constexpr int TD_MMA_WARPS = 2;   // 2: one per M tile; 4: (M tile) x (stage parity)
