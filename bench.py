@@ -388,6 +388,29 @@ def measure_switch(layers, meta, cfg, device, T=16, events=8, steps_between=8):
         res[mode_name] = {"layers": n, "tokens": T, "stack_step_ms": sm, "tokens_per_s": T / (sm / 1e3),
                           "switch_event_device_ms": dm, "switch_event_host_ms": hm,
                           "switch_fraction_of_step": dm / sm, "events": events}
+    # device-side selection: statistics collected during the forwards, then per layer one call that ranks the cached
+    # channels and rewrites the tables (it synchronises to bring the chosen sets back to the host mirror)
+    for l in layers:
+        l.set_stats_collection(True)
+    for _ in range(3):
+        stack_step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps_between):
+        stack_step()
+    e1.record()
+    torch.cuda.synchronize()
+    step_stats_ms = e0.elapsed_time(e1) / steps_between
+    t0 = time.perf_counter()
+    for l in layers:
+        l.select_significant(cfg.max_sig, reset=True)
+    sel_host_ms = (time.perf_counter() - t0) * 1e3
+    for l in layers:
+        l.set_stats_collection(False)
+    binding.set_channel_switch_many(layers, [m["sets"] for m in meta])
+    res["device_selection"] = {"layers": n, "tokens": T, "stack_step_ms_with_stats": step_stats_ms,
+                               "select_all_layers_host_ms": sel_host_ms}
     return res
 
 

@@ -191,6 +191,28 @@ dynamo_status dynamo_poll_status(dynamo_ctx* ctx, void* stream);
  * 0 switches the tcgen05 path off.  Both paths implement the same arithmetic definition. */
 dynamo_status dynamo_set_tc_min_rows(dynamo_ctx* ctx, int32_t rows);
 
+/* Runtime selection of the significant channels on the device (Sections IV-B, V-A: the channels whose dynamics
+ * are most prominent under the current data are the ones to switch; only cached channels can be raised).
+ *
+ * dynamo_set_stats_collection(on): while on, every forward also accumulates, per routed expert e and cached
+ *   channel c, A[e][c] += sum over the tokens routed to e in that forward of |x[t][c]| -- in fp32, tokens in
+ *   ascending order inside a forward and ONE addition of the forward's sum to the running total, so the statistics
+ *   are reproducible bit for bit (they decide an integer selection).  One extra kernel per forward.  The paper
+ *   leaves the statistic open ("significance of channel weights ... corresponding to the tokens"); the activation
+ *   mass of the input channel is the reading taken here.
+ * dynamo_get_channel_stats: copies A to stats_out, DEVICE fp32 [E, P] (column j = cached channel cache_idx[e][j]).
+ * dynamo_select_significant: per expert with base bits < 8 the n_select (<= max_sig, <= P) cached channels with
+ *   the largest A, ties -> lower channel index, become the significant set (slot order = rank order); 8-bit
+ *   experts get the empty set.  The tables are rewritten by a device kernel exactly as dynamo_set_channel_switch
+ *   would write them; the call then SYNCHRONISES the stream to bring the chosen sets back (host mirror, and
+ *   sig_idx_out host [E, max_sig] padded with -1 / sig_cnt_out host [E] if not NULL).  reset != 0 zeroes A.
+ * Errors: NULL ctx -> ERR_NULL; before pack -> ERR_STATE; n_select out of range or a pool too large to rank in
+ * shared memory (P > 12288) -> ERR_SHAPE. */
+dynamo_status dynamo_set_stats_collection(dynamo_ctx* ctx, int32_t on);
+dynamo_status dynamo_get_channel_stats(dynamo_ctx* ctx, float* stats_out, void* stream);
+dynamo_status dynamo_select_significant(dynamo_ctx* ctx, int32_t n_select, int32_t reset, int32_t* sig_idx_out,
+                                        int32_t* sig_cnt_out, void* stream);
+
 /* Which kernel serves small batches (forwards of at most 64 tokens, where every expert has few rows and the
  * forward is bound by streaming the packed weights of Section V-B from HBM):
  *   DYNAMO_DECODE_STREAM (default): the streaming kernel (mma.sync) takes every expert, as it does for the

@@ -300,3 +300,37 @@ class OracleLayer:
                 acc = acc + sh[i]
             y[t] = acc
         return {"idx": idx, "w": w, "offsets": offsets, "perm": perm, "y": y}
+
+
+# ---- runtime selection of the significant channels (Sections IV-B, V-A; a "next" row of the scope table) ----
+# The statistic decides an integer (which channels are selected), so it is accumulated in the CUDA path's
+# precision and order: float32, tokens ascending inside a forward, then one float32 addition to the running total.
+
+def channel_stats_update(stats: np.ndarray, x_u16: np.ndarray, idx: np.ndarray, pool: np.ndarray) -> np.ndarray:
+    """stats float32 [E, P] += per expert e, cached channel pool[e][j]: sum over the tokens routed to e (ascending)
+    of |x[t][pool[e][j]]|.  x_u16: bf16 bit patterns [T, d]; idx: int32 [T, k] chosen experts; returns stats."""
+    E, P = pool.shape
+    xa = np.abs((x_u16.astype(np.uint32) << 16).view(np.float32))      # |x| as float32: exact for bf16
+    out = np.array(stats, dtype=np.float32, copy=True)
+    for e in range(E):
+        toks = np.flatnonzero((idx == e).any(axis=1))                   # ascending token order
+        if len(toks) == 0:
+            continue
+        batch = np.zeros((P,), dtype=np.float32)
+        for t in toks:
+            batch = (batch + xa[t, pool[e]]).astype(np.float32)         # one rounding per addition, in token order
+        out[e] = (out[e] + batch).astype(np.float32)
+    return out
+
+
+def select_significant(stats: np.ndarray, pool: np.ndarray, n_select: int, switchable: Sequence[bool]):
+    """Per expert: the n_select cached channels with the largest statistic, ties -> lower channel index, in rank
+    order; experts that are not switchable (8-bit base) get the empty set."""
+    sets = []
+    for e in range(pool.shape[0]):
+        if not switchable[e]:
+            sets.append(np.zeros((0,), np.int32))
+            continue
+        order = sorted(range(pool.shape[1]), key=lambda j: (-float(stats[e, j]), int(pool[e, j])))
+        sets.append(np.array([pool[e, j] for j in order[: min(n_select, pool.shape[1])]], dtype=np.int32))
+    return sets

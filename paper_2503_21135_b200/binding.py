@@ -33,7 +33,8 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_BITS", "ERR_ALIGN", "ERR_ARE
 EXPORTED = ["dynamo_create", "dynamo_destroy", "dynamo_arena_bytes", "dynamo_pack_experts",
             "dynamo_set_channel_switch", "dynamo_set_channel_switch_many", "dynamo_set_switch_mode",
             "dynamo_moe_forward", "dynamo_moe_forward_router", "dynamo_moe_forward_host", "dynamo_export_codes", "dynamo_expert_stream_bytes",
-            "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_decode_kernel", "dynamo_set_prefill_kernel", "dynamo_route_permute_static", "dynamo_kernel_launches", "dynamo_status_str"]
+            "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_decode_kernel", "dynamo_set_prefill_kernel", "dynamo_set_stats_collection",
+            "dynamo_get_channel_stats", "dynamo_select_significant", "dynamo_route_permute_static", "dynamo_kernel_launches", "dynamo_status_str"]
 
 
 class LayerDesc(ctypes.Structure):
@@ -80,6 +81,9 @@ def load():
         L.dynamo_set_tc_min_rows.argtypes = [vp, i32]
         L.dynamo_set_decode_kernel.argtypes = [vp, i32]
         L.dynamo_set_prefill_kernel.argtypes = [vp, i32]
+        L.dynamo_set_stats_collection.argtypes = [vp, i32]
+        L.dynamo_get_channel_stats.argtypes = [vp, vp, vp]
+        L.dynamo_select_significant.argtypes = [vp, i32, i32, i32p, i32p, vp]
         L.dynamo_route_permute_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
         L.dynamo_kernel_launches.argtypes = [vp]
         L.dynamo_kernel_launches.restype = ctypes.c_int64
@@ -340,6 +344,24 @@ class DynamoLayer:
 
     def set_tc_min_rows(self, rows: int):
         _check(dynamo_set_tc_min_rows(self.ctx, rows), "dynamo_set_tc_min_rows")
+
+    def set_stats_collection(self, on: bool):
+        _check(load().dynamo_set_stats_collection(self.ctx, int(bool(on))), "dynamo_set_stats_collection")
+
+    def channel_stats(self) -> torch.Tensor:
+        """Accumulated activation mass fp32 [E, P] (column j = cached channel cache_idx[e][j])."""
+        out = torch.empty((self.desc.n_experts, self.desc.cache_size), dtype=torch.float32, device=self.device)
+        _check(load().dynamo_get_channel_stats(self.ctx, out.data_ptr(), _stream()), "dynamo_get_channel_stats")
+        return out
+
+    def select_significant(self, n_select: int, reset: bool = True):
+        """Install, per expert, the n_select cached channels with the largest statistics; returns the sets."""
+        E, S = self.desc.n_experts, self.desc.max_sig
+        idx = np.full((E, max(S, 1)), -1, dtype=np.int32)
+        cnt = np.zeros((E,), dtype=np.int32)
+        _check(load().dynamo_select_significant(self.ctx, n_select, int(bool(reset)), _i32p(idx), _i32p(cnt), _stream()),
+               "dynamo_select_significant")
+        return [idx[e, : cnt[e]].copy() for e in range(E)]
 
     def set_prefill_kernel(self, kind: int):
         _check(dynamo_set_prefill_kernel(self.ctx, kind), "dynamo_set_prefill_kernel")

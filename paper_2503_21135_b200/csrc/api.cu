@@ -31,6 +31,9 @@ cudaError_t launch_ffn_tc2(const LayerDev* L, const WsDev& ws, int gateup, int n
                            cudaStream_t st);
 cudaError_t launch_ffn_tcd(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int ksplit, int n_experts,
                            long long split_stride, int n_sms, cudaStream_t st);
+cudaError_t launch_stats(const LayerDev* L, const WsDev& ws, const void* x, float* stats, int E, cudaStream_t st);
+cudaError_t launch_select(const LayerDev* L, float* stats, int E, int P, int n_sel, int reset, int32_t* chosen,
+                          cudaStream_t st);
 cudaError_t launch_switch(const SwitchLayers& layers, int n_layers, int E, const int32_t* staging, int per_layer_ints,
                           cudaStream_t st);
 }  // namespace dyn
@@ -51,7 +54,7 @@ inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
 struct ArenaLayout {
     size_t header = 0;
     std::vector<size_t> w13, w2, s8m8_g, s8m8_u, q8_g, q8_u, cw_g, cw_u, pool_hi;
-    size_t cache_idx = 0, sig_chan = 0, sig_pool = 0, sig_cnt = 0, sigmask = 0;
+    size_t cache_idx = 0, sig_chan = 0, sig_pool = 0, sig_cnt = 0, sigmask = 0, stats = 0;
     size_t total = 0;
 };
 
@@ -127,6 +130,7 @@ void arena_layout(const dynamo_layer_desc& D, const int32_t* bits, ArenaLayout& 
     A.sig_pool = take((size_t)D.n_experts * S_pad * 4);
     A.sig_cnt = take((size_t)D.n_experts * 4);
     A.sigmask = take((size_t)D.n_experts * (d / 32) * 4);
+    A.stats = take((size_t)D.n_experts * ((P + 31) / 32 * 32) * 4);  // activation mass per (expert, cached channel)
     A.total = off;
 }
 
@@ -176,6 +180,7 @@ struct dynamo_ctx {
     int switch_mode = DYNAMO_SWITCH_SELECT;
     int tc_min_rows = TC_MIN_ROWS;               // experts with more rows take the tcgen05 path
     int decode_kernel = DYNAMO_DECODE_STREAM;
+    int collect_stats = 0;                       // 1: every forward adds to the per-channel activation statistics
     int prefill_kernel = DYNAMO_PREFILL_PAIR;    // which tcgen05 kernel serves experts above the row threshold    // which kernel serves forwards of up to DECODE_FOLD_TOKENS tokens
     int n_sms = 148;                             // SM count of the device the layer was packed on
     int64_t launches = 0;
@@ -320,6 +325,50 @@ dynamo_status dynamo_set_tc_min_rows(dynamo_ctx* ctx, int32_t rows) {
     if (rows < 0) return DYNAMO_ERR_SHAPE;
     // the streaming path handles one 32-token chunk per expert when both paths are active
     ctx->tc_min_rows = rows == 0 ? 0x7fffffff : (rows < TC_MIN_ROWS ? rows : TC_MIN_ROWS);
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_set_stats_collection(dynamo_ctx* ctx, int32_t on) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    ctx->collect_stats = on ? 1 : 0;
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_get_channel_stats(dynamo_ctx* ctx, float* stats_out, void* stream) {
+    if (!ctx || !stats_out) return DYNAMO_ERR_NULL;
+    if (!ctx->packed) return DYNAMO_ERR_STATE;
+    const dynamo_layer_desc& D = ctx->D;
+    const size_t P = D.cache_size, P_pad = (P + 31) / 32 * 32;
+    CUDA_TRY(cudaMemcpy2DAsync(stats_out, P * 4, ctx->arena + ctx->A.stats, P_pad * 4, P * 4, D.n_experts,
+                               cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_select_significant(dynamo_ctx* ctx, int32_t n_select, int32_t reset, int32_t* sig_idx_out,
+                                        int32_t* sig_cnt_out, void* stream) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    if (!ctx->packed) return DYNAMO_ERR_STATE;
+    const dynamo_layer_desc& D = ctx->D;
+    if (n_select < 0 || n_select > D.max_sig) return DYNAMO_ERR_SHAPE;
+    if ((size_t)D.cache_size * 4 > 48 * 1024) return DYNAMO_ERR_SHAPE;  // the ranking keeps a pool's statistics in shared memory
+    cudaStream_t st = (cudaStream_t)stream;
+    const int E = D.n_experts, S_pad = s_pad_of(D);
+    int32_t* chosen = (int32_t*)(ctx->ws + ctx->W.stage_switch);
+    CUDA_TRY(launch_select((const LayerDev*)ctx->arena, (float*)(ctx->arena + ctx->A.stats), E, D.cache_size, n_select,
+                           reset ? 1 : 0, chosen, st));
+    ctx->launches += 1;
+    // the host mirror of the sets (stream bytes, exports, later validation) follows the device's choice
+    std::vector<int32_t> host((size_t)E * S_pad);
+    CUDA_TRY(cudaMemcpyAsync(host.data(), chosen, host.size() * 4, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    for (int e = 0; e < E; ++e) {
+        std::vector<int32_t>& lst = ctx->sig[e];
+        lst.clear();
+        for (int j = 0; j < S_pad && host[(size_t)e * S_pad + j] >= 0; ++j) lst.push_back(host[(size_t)e * S_pad + j]);
+        if (sig_cnt_out) sig_cnt_out[e] = (int32_t)lst.size();
+        if (sig_idx_out)
+            for (int j = 0; j < D.max_sig; ++j) sig_idx_out[(size_t)e * D.max_sig + j] = j < (int)lst.size() ? lst[j] : -1;
+    }
     return DYNAMO_OK;
 }
 
@@ -557,6 +606,10 @@ static dynamo_status forward_impl(dynamo_ctx* ctx, const void* x, const float* r
         CUDA_TRY(launch_route(router_logits, T, D.n_experts, D.top_k, D.renormalize, ws.topk_idx, ws.topk_w, st));
     CUDA_TRY(launch_scan(ws, D.n_experts, D.n_shared, D.top_k, st));
     CUDA_TRY(launch_gather(L, ws, x, st));
+    if (ctx->collect_stats) {
+        CUDA_TRY(launch_stats(L, ws, x, (float*)(ctx->arena + ctx->A.stats), D.n_experts, st));
+        ctx->launches += 1;
+    }
     const bool use_tc = ws.tc_min != 0x7fffffff;                  // experts above 32 rows take the tcgen05 path
     const long long split_stride = (long long)ws.Rpad * D.d_model;  // partials of one K split: [Rpad][d]
     if (ws.fold) {

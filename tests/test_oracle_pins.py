@@ -391,3 +391,50 @@ def test_router_scores_match_library_matmul_and_closed_forms():
     xs = bf16_bits(np.array([[1.0, 2.0, -3.0, 0.5]]))
     ws = bf16_bits(np.array([[1.0, 0.0, 0.0, 0.0], [0.5, 0.5, 0.5, 0.5]]))
     assert oracle.router_scores(xs, ws, np.array([0.0, 1.0], np.float32)).tolist() == [[1.0, 1.25]]
+
+
+# ---- runtime selection of the significant channels ---------------------------------------------
+
+def test_channel_stats_closed_forms_and_order():
+    rng = np.random.default_rng(5)
+    T, d, E, k, P = 40, 64, 4, 2, 8
+    idx = np.stack([rng.permutation(E)[:k] for _ in range(T)]).astype(np.int32)
+    pool = np.stack([np.sort(rng.permutation(d)[:P]) for _ in range(E)]).astype(np.int32)
+    # |x| = 1 everywhere: the statistic is the number of tokens routed to the expert (exact in float32)
+    ones = bf16_bits(np.where(rng.random((T, d)) < 0.5, 1.0, -1.0))
+    s = oracle.channel_stats_update(np.zeros((E, P), np.float32), ones, idx, pool)
+    assert np.array_equal(s, np.tile(np.bincount(idx.ravel(), minlength=E).astype(np.float32)[:, None], (1, P)))
+    # x zero outside one channel: only that channel (where cached) accumulates, by the routed tokens' |x|
+    xz = np.zeros((T, d))
+    xz[:, pool[1, 3]] = rng.integers(1, 5, size=T)                    # small integers: sums exact
+    s = oracle.channel_stats_update(np.zeros((E, P), np.float32), bf16_bits(xz), idx, pool)
+    for e in range(E):
+        toks = (idx == e).any(axis=1)
+        expect = np.where(pool[e] == pool[1, 3], xz[toks, pool[1, 3]].sum(), 0.0)
+        assert np.array_equal(s[e], expect.astype(np.float32))
+    # two updates add: running total = first + second (integers: no rounding)
+    s2 = oracle.channel_stats_update(s, bf16_bits(xz), idx, pool)
+    assert np.array_equal(s2, 2 * s)
+    # float32, token-ascending order: 2^24 + 1 + 1 stays 2^24 in that order (a float64 or reordered sum would not)
+    big = np.zeros((3, d))
+    big[0, pool[0, 0]], big[1, pool[0, 0]], big[2, pool[0, 0]] = 2.0 ** 24, 1.0, 1.0
+    s3 = oracle.channel_stats_update(np.zeros((E, P), np.float32), bf16_bits(big), np.zeros((3, 1), np.int32), pool)
+    assert s3[0, 0] == np.float32(2.0 ** 24)
+
+
+def test_select_significant_rank_rule():
+    pool = np.array([[2, 5, 9, 11, 30, 31], [0, 1, 2, 3, 4, 5]], np.int32)
+    stats = np.array([[1.0, 7.0, 7.0, 0.0, 3.0, 9.0], [0.0, 0.0, 0.0, 0.0, 0.0, 0.0]], np.float32)
+    sets = oracle.select_significant(stats, pool, 4, [True, True])
+    # hand-ranked: 9.0 (ch 31), then the tie 7.0 -> lower channel first (5 before 9), then 3.0 (ch 30)
+    assert sets[0].tolist() == [31, 5, 9, 30]
+    assert sets[1].tolist() == [0, 1, 2, 3]                             # all equal: lowest channels
+    assert oracle.select_significant(stats, pool, 4, [False, True])[0].tolist() == []
+    assert len(oracle.select_significant(stats, pool, 10, [True, True])[0]) == 6   # never more than the pool holds
+    # distinct values: equals a library argsort; and nothing left out beats anything selected
+    rng = np.random.default_rng(3)
+    st = rng.permutation(64).astype(np.float32).reshape(1, 64)
+    pl = np.arange(64, dtype=np.int32).reshape(1, 64) * 3
+    got = oracle.select_significant(st, pl, 10, [True])[0]
+    assert got.tolist() == (pl[0][np.argsort(-st[0], kind="stable")[:10]]).tolist()
+    assert st[0][np.isin(pl[0], got)].min() > st[0][~np.isin(pl[0], got)].max()
