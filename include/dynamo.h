@@ -191,6 +191,17 @@ dynamo_status dynamo_poll_status(dynamo_ctx* ctx, void* stream);
  * 0 switches the tcgen05 path off.  Both paths implement the same arithmetic definition. */
 dynamo_status dynamo_set_tc_min_rows(dynamo_ctx* ctx, int32_t rows);
 
+/* Precision the significant channels are served at (Section IV-B: once the original channels are back in place
+ * they are requantized to the precision the new data calls for, which may be higher or lower than before).
+ *   hi_bits : host int32 [E], each in {2, 3, 4, 6, 8}; 8 for every expert after dynamo_pack_experts.
+ * For every routed expert with base bits < 8 whose value changes, one kernel recomputes from the stored group
+ * extrema the parameters of the expert's uniform hi_bits[e]-bit quantization of W_gate and W_up (same groups, same
+ * quantizer as pack), and from the bf16 channel cache the codes and forward-ready values of all cached channels.
+ * A significant channel c then takes the value it has in that quantization; the sets themselves are unchanged.
+ * Entries of 8-bit experts are checked but ignored.  Stream-ordered.
+ * Errors: NULL -> ERR_NULL; before pack -> ERR_STATE; a value outside the list -> ERR_BITS (nothing changes). */
+dynamo_status dynamo_set_channel_precision(dynamo_ctx* ctx, const int32_t* hi_bits, void* stream);
+
 /* Runtime selection of the significant channels on the device (Sections IV-B, V-A: the channels whose dynamics
  * are most prominent under the current data are the ones to switch; only cached channels can be raised).
  *

@@ -227,6 +227,16 @@ class OracleLayer:
                 self.hi[e] = tuple(QuantMatrix(*quantize(w[e], G, HI_BITS)) for w in (w_gate, w_up))
         self.sig: List[np.ndarray] = [np.zeros((0,), np.int32) for _ in range(self.E)]
 
+    def set_channel_precision(self, hi_bits: Sequence[int], w_gate, w_up) -> None:
+        """Precision the significant channels are served at, per routed expert (Section IV-B: the replaced
+        channels are requantized to the precision the new data calls for): a significant channel of expert e
+        takes the value it has in the expert's uniform hi_bits[e]-bit quantization of the ORIGINAL W_gate / W_up
+        (same groups, same quantizer).  w_gate, w_up: the original bf16 bit patterns [E+Es, f, d]."""
+        assert len(hi_bits) == self.E
+        for e in range(self.E):
+            if self.hi[e] is not None:
+                self.hi[e] = tuple(QuantMatrix(*quantize(w[e], self.G, int(hi_bits[e]))) for w in (w_gate, w_up))
+
     def set_channel_switch(self, sets: Sequence[np.ndarray]) -> None:
         """Install the significant-channel set of every routed expert (state depends only on it)."""
         assert len(sets) == self.E

@@ -33,7 +33,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_BITS", "ERR_ALIGN", "ERR_ARE
 EXPORTED = ["dynamo_create", "dynamo_destroy", "dynamo_arena_bytes", "dynamo_pack_experts",
             "dynamo_set_channel_switch", "dynamo_set_channel_switch_many", "dynamo_set_switch_mode",
             "dynamo_moe_forward", "dynamo_moe_forward_router", "dynamo_moe_forward_host", "dynamo_export_codes", "dynamo_expert_stream_bytes",
-            "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_decode_kernel", "dynamo_set_prefill_kernel", "dynamo_set_stats_collection",
+            "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_decode_kernel", "dynamo_set_prefill_kernel", "dynamo_set_stats_collection", "dynamo_set_channel_precision",
             "dynamo_get_channel_stats", "dynamo_select_significant", "dynamo_route_permute_static", "dynamo_kernel_launches", "dynamo_status_str"]
 
 
@@ -82,6 +82,7 @@ def load():
         L.dynamo_set_decode_kernel.argtypes = [vp, i32]
         L.dynamo_set_prefill_kernel.argtypes = [vp, i32]
         L.dynamo_set_stats_collection.argtypes = [vp, i32]
+        L.dynamo_set_channel_precision.argtypes = [vp, i32p, vp]
         L.dynamo_get_channel_stats.argtypes = [vp, vp, vp]
         L.dynamo_select_significant.argtypes = [vp, i32, i32, i32p, i32p, vp]
         L.dynamo_route_permute_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
@@ -344,6 +345,12 @@ class DynamoLayer:
 
     def set_tc_min_rows(self, rows: int):
         _check(dynamo_set_tc_min_rows(self.ctx, rows), "dynamo_set_tc_min_rows")
+
+    def set_channel_precision(self, hi_bits):
+        """Precision the significant channels of each routed expert are served at: int [E], each in {2,3,4,6,8}."""
+        hb = np.ascontiguousarray(np.asarray(hi_bits, dtype=np.int32))
+        assert hb.shape == (self.desc.n_experts,)
+        _check(load().dynamo_set_channel_precision(self.ctx, _i32p(hb), _stream()), "dynamo_set_channel_precision")
 
     def set_stats_collection(self, on: bool):
         _check(load().dynamo_set_stats_collection(self.ctx, int(bool(on))), "dynamo_set_stats_collection")

@@ -13,6 +13,7 @@ cudaError_t launch_pack_blocks(const void* src_a, const void* src_b, int n_rows_
 cudaError_t launch_pack_hi(const void* w_gate, const void* w_up, int f, int d, int G, int P,
                            const int32_t* cache_idx_dev, const ExpertDev& ex, cudaStream_t st);
 cudaError_t launch_requant(const LayerDev* L, int f, const int32_t* items_dev, int n_items, cudaStream_t st);
+cudaError_t launch_retarget(LayerDev* L, int e, int f, int bits, cudaStream_t st);
 cudaError_t launch_export(const LayerDev* L, int e, int mat, int which, long long n_elems, uint8_t* q, uint16_t* sc,
                           uint16_t* zr, cudaStream_t st);
 cudaError_t launch_route(const float* logits, int T, int E, int k, int renorm, int32_t* idx, float* w,
@@ -53,7 +54,7 @@ inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct ArenaLayout {
     size_t header = 0;
-    std::vector<size_t> w13, w2, s8m8_g, s8m8_u, q8_g, q8_u, cw_g, cw_u, pool_hi;
+    std::vector<size_t> w13, w2, s8m8_g, s8m8_u, mm_g, mm_u, q8_g, q8_u, cw_g, cw_u, pool_hi;
     size_t cache_idx = 0, sig_chan = 0, sig_pool = 0, sig_cnt = 0, sigmask = 0, stats = 0;
     size_t total = 0;
 };
@@ -108,6 +109,7 @@ void arena_layout(const dynamo_layer_desc& D, const int32_t* bits, ArenaLayout& 
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
     A.w13.assign(n, 0); A.w2.assign(n, 0);
     A.s8m8_g.assign(n, 0); A.s8m8_u.assign(n, 0); A.q8_g.assign(n, 0); A.q8_u.assign(n, 0);
+    A.mm_g.assign(n, 0); A.mm_u.assign(n, 0);
     A.cw_g.assign(n, 0); A.cw_u.assign(n, 0); A.pool_hi.assign(n, 0);
     for (int e = 0; e < n; ++e) {
         const size_t blk = block_bytes(bits[e], (int)G);
@@ -118,6 +120,8 @@ void arena_layout(const dynamo_layer_desc& D, const int32_t* bits, ArenaLayout& 
         if (bits[e] >= HI_BITS) continue;
         A.s8m8_g[e] = take(f * (d / G) * 4);
         A.s8m8_u[e] = take(f * (d / G) * 4);
+        A.mm_g[e] = take(f * (d / G) * 4);
+        A.mm_u[e] = take(f * (d / G) * 4);
         A.q8_g[e] = take(P * f);
         A.q8_u[e] = take(P * f);
         A.cw_g[e] = take(P * f * 2);
@@ -170,6 +174,7 @@ struct dynamo_ctx {
     dynamo_layer_desc D;
     bool packed = false;
     std::vector<int32_t> bits;
+    std::vector<int32_t> hi_bits;                // precision the significant channels of each routed expert are served at
     std::vector<int32_t> cache_idx;              // host copy [E][P]
     std::vector<std::vector<int32_t>> sig;       // current sets, in slot order
     ArenaLayout A;
@@ -328,6 +333,25 @@ dynamo_status dynamo_set_tc_min_rows(dynamo_ctx* ctx, int32_t rows) {
     return DYNAMO_OK;
 }
 
+dynamo_status dynamo_set_channel_precision(dynamo_ctx* ctx, const int32_t* hi_bits, void* stream) {
+    if (!ctx || !hi_bits) return DYNAMO_ERR_NULL;
+    if (!ctx->packed) return DYNAMO_ERR_STATE;
+    const dynamo_layer_desc& D = ctx->D;
+    for (int e = 0; e < D.n_experts; ++e) {
+        const int b = hi_bits[e];
+        if (b != 2 && b != 3 && b != 4 && b != 6 && b != 8) return DYNAMO_ERR_BITS;  // nothing changes on an error
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    for (int e = 0; e < D.n_experts; ++e) {
+        if (ctx->bits[e] >= HI_BITS || ctx->hi_bits[e] == hi_bits[e]) continue;  // 8-bit experts have no cache pool
+        CUDA_TRY(launch_retarget((LayerDev*)ctx->arena, e, D.d_ff, hi_bits[e], st));
+        ctx->hi_bits[e] = hi_bits[e];
+        ctx->host_layer.ex[e].hi_bits = hi_bits[e];
+        ctx->launches += 1;
+    }
+    return DYNAMO_OK;
+}
+
 dynamo_status dynamo_set_stats_collection(dynamo_ctx* ctx, int32_t on) {
     if (!ctx) return DYNAMO_ERR_NULL;
     ctx->collect_stats = on ? 1 : 0;
@@ -420,6 +444,7 @@ dynamo_status dynamo_pack_experts(dynamo_ctx* ctx, const void* w_gate, const voi
     ctx->arena = (uint8_t*)weights_arena;
     ctx->ws = (uint8_t*)workspace;
     ctx->bits.assign(bits, bits + n);
+    ctx->hi_bits.assign(D.n_experts, HI_BITS);
     ctx->cache_idx.assign(cache_idx, cache_idx + (size_t)D.n_experts * P);
     ctx->sig.assign(D.n_experts, {});
 
@@ -449,9 +474,12 @@ dynamo_status dynamo_pack_experts(dynamo_ctx* ctx, const void* w_gate, const voi
         x.w13 = base + A.w13[e];
         x.w2 = base + A.w2[e];
         x.switchable = (e < D.n_experts && bits[e] < HI_BITS) ? 1 : 0;
+        x.hi_bits = HI_BITS;
         if (x.switchable) {
             x.s8m8[0] = (uint32_t*)(base + A.s8m8_g[e]);
             x.s8m8[1] = (uint32_t*)(base + A.s8m8_u[e]);
+            x.gminmax[0] = (uint32_t*)(base + A.mm_g[e]);
+            x.gminmax[1] = (uint32_t*)(base + A.mm_u[e]);
             x.pool_q8[0] = base + A.q8_g[e];
             x.pool_q8[1] = base + A.q8_u[e];
             x.cache_w[0] = (__nv_bfloat16*)(base + A.cw_g[e]);

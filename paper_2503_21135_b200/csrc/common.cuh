@@ -24,13 +24,14 @@ struct ExpertDev {
     const uint8_t* w13;        // packed blocks of the fused gate/up matrix: [n_rb13][n_kc13][blk_bytes]
     const uint8_t* w2;         // packed blocks of the down matrix:          [n_rb2][n_kc2][blk_bytes]
     __half* pool_hi;           // [n_rb13][P + 1][256] fp16, value s8*q8+m8 of cached channel p (tile P = zeros)
-    uint32_t* s8m8[2];         // gate, up: [f][d/G] half2 {scale, zero} of the 8-bit quantization
+    uint32_t* s8m8[2];         // gate, up: [f][d/G] half2 {scale, zero} of the high-precision (hi_bits) quantization
+    uint32_t* gminmax[2];      // gate, up: [f][d/G] bf16 pair {min, max} of every group of the original weights
     uint8_t* pool_q8[2];       // gate, up: [P][f] 8-bit codes of the cached channels
     __nv_bfloat16* cache_w[2]; // gate, up: [P][f] bf16 originals of the cached channels (the channel cache)
     int32_t bits;
     int32_t blk_bytes;         // bytes of one packed block (codes + params)
     int32_t switchable;        // routed expert with bits < 8
-    int32_t pad_;
+    int32_t hi_bits;           // precision the significant channels are served at (8 after pack; retargetable)
 };
 
 struct LayerDev {

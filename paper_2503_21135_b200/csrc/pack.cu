@@ -98,11 +98,15 @@ __global__ void pack_hi_kernel(const __nv_bfloat16* __restrict__ w_gate, const _
     int pi = 0;
     for (int g = 0; g < ng; ++g) {
         double lo = bf16_to_double(row[g * G]), hi = lo;
+        __nv_bfloat16 lo_b = row[g * G], hi_b = lo_b;
         for (int i = 1; i < G; ++i) {
             double v = bf16_to_double(row[g * G + i]);
-            lo = v < lo ? v : lo;
-            hi = v > hi ? v : hi;
+            if (v < lo) { lo = v; lo_b = row[g * G + i]; }
+            if (v > hi) { hi = v; hi_b = row[g * G + i]; }
         }
+        // the group's extrema stay with the cache: a later change of the target precision needs them
+        ex.gminmax[mat][(long long)n * ng + g] =
+            (uint32_t)__bfloat16_as_ushort(lo_b) | ((uint32_t)__bfloat16_as_ushort(hi_b) << 16);
         __half s_h, m_h;
         double s, m;
         group_params(lo, hi, HI_BITS, s_h, m_h, s, m);
@@ -140,10 +144,43 @@ __global__ void requant_from_cache_kernel(const LayerDev* __restrict__ L, const 
     const __half2 pr = *reinterpret_cast<const __half2*>(&prw);
     const double s = (double)__low2float(pr), m = (double)__high2float(pr);
     const __nv_bfloat16 w = ex.cache_w[mat][(long long)p * L->f + n];
-    const int q = quantize_code(bf16_to_double(w), s, m, HI_BITS);
+    const int q = quantize_code(bf16_to_double(w), s, m, ex.hi_bits);
     ex.pool_q8[mat][(long long)p * L->f + n] = (uint8_t)q;
     const int rb = n >> 7, rib = w13_row_in_block(n, mat);
     ex.pool_hi[pool_tile_off(rb, p, L->P_pad) / 2 + rib] = __double2half(s * (double)q + m);
+}
+
+// Change the precision the cached channels of expert e are served at (Section IV-B: after replacement the
+// original channels are requantized to the precision the new data calls for, higher or lower than before):
+// the parameters of every group at `bits` from the stored group extrema, then code and forward-ready value of
+// every cached channel from its bf16 original.  One thread per row n of one matrix (grid.y: gate, up).
+__global__ void retarget_kernel(LayerDev* __restrict__ L, int e, int bits) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    const int mat = blockIdx.y;
+    ExpertDev& ex = L->ex[e];
+    if (n == 0 && mat == 0) ex.hi_bits = bits;
+    if (n >= L->f) return;
+    const int ng = L->d / L->G, G = L->G, P = L->P, f = L->f;
+    const int32_t* ci = L->cache_idx + (long long)e * P;
+    const int rb = n >> 7, rib = w13_row_in_block(n, mat);
+    int pi = 0;
+    for (int g = 0; g < ng; ++g) {
+        const uint32_t mm = ex.gminmax[mat][(long long)n * ng + g];
+        const double lo = bf16_to_double(__ushort_as_bfloat16((unsigned short)(mm & 0xffff)));
+        const double hi = bf16_to_double(__ushort_as_bfloat16((unsigned short)(mm >> 16)));
+        __half s_h, m_h;
+        double s, m;
+        group_params(lo, hi, bits, s_h, m_h, s, m);
+        __half2 pr = __halves2half2(s_h, m_h);
+        ex.s8m8[mat][(long long)n * ng + g] = *reinterpret_cast<uint32_t*>(&pr);
+        while (pi < P && ci[pi] < (g + 1) * G) {
+            const __nv_bfloat16 w = ex.cache_w[mat][(long long)pi * f + n];
+            const int q = quantize_code(bf16_to_double(w), s, m, bits);
+            ex.pool_q8[mat][(long long)pi * f + n] = (uint8_t)q;
+            ex.pool_hi[pool_tile_off(rb, pi, L->P_pad) / 2 + rib] = __double2half(s * (double)q + m);
+            ++pi;
+        }
+    }
 }
 
 // Export logical codes and params.  One thread per (n, k).
@@ -222,6 +259,12 @@ cudaError_t launch_pack_hi(const void* w_gate, const void* w_up, int f, int d, i
     dim3 grid((f + 127) / 128, 2);
     pack_hi_kernel<<<grid, 128, 0, st>>>((const __nv_bfloat16*)w_gate, (const __nv_bfloat16*)w_up, f, d, G, P,
                                          cache_idx_dev, ex);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_retarget(LayerDev* L, int e, int f, int bits, cudaStream_t st) {
+    dim3 grid((f + 127) / 128, 2);
+    retarget_kernel<<<grid, 128, 0, st>>>(L, e, bits);
     return cudaGetLastError();
 }
 

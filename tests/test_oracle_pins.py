@@ -65,7 +65,7 @@ def test_bf16_decode_matches_torch():
 
 # ---- C1 quantizer ------------------------------------------------------------------------
 
-@pytest.mark.parametrize("bits", [2, 3, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 6, 8])
 @pytest.mark.parametrize("G", [64, 128])
 def test_quantizer_bruteforce_nearest_level(bits, G):
     rng = np.random.default_rng(100 + bits + G)
@@ -99,7 +99,7 @@ def test_quantizer_bruteforce_nearest_level(bits, G):
                 assert abs(v - levels[code]) <= bound
 
 
-@pytest.mark.parametrize("bits", [2, 3, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 6, 8])
 def test_quantizer_lossless_construction_and_ties(bits):
     # group = m + j*s with s a power of two and m fp16-exact  =>  q = j and s*q+m = w exactly
     G, L = 64, 2 ** bits - 1
@@ -333,6 +333,31 @@ def test_all_channels_switched_equals_uniform_8bit():
         ref.base[e] = (ref.base[e][0], ref.base[e][1], layer.base[e][2])
     layer.set_channel_switch([np.arange(layer.d)] * 4)
     assert np.array_equal(layer.forward(x, logits)["y"], ref.forward(x, logits)["y"])
+
+
+@pytest.mark.parametrize("hb", [3, 4, 6])
+def test_channel_precision_all_switched_equals_uniform_target(hb):
+    # with every channel significant and target precision hb, gate/up are the expert's uniform hb-bit
+    # quantization; a target equal to the base bit-width changes nothing; going back to 8 restores the state
+    layer, x, logits, (wg, wu, wd) = _tiny_layer(seed=5, bits=(2, 3, 2, 8))
+    ug, uu = bf16_bits(wg), bf16_bits(wu)
+    layer.set_channel_switch([np.arange(0, layer.d, 3)] * 4)
+    y8 = layer.forward(x, logits)["y"]
+    layer.set_channel_precision([hb] * 4, ug, uu)
+    ref = oracle.OracleLayer(ug, uu, bf16_bits(wd), [hb, hb, hb, 8], layer.G, 4, 2)
+    for e in range(3):
+        ref.base[e] = (ref.base[e][0], ref.base[e][1], layer.base[e][2])
+    assert layer.hi[3] is None                                   # the 8-bit expert has no switch
+    layer.set_channel_switch([np.arange(layer.d)] * 4)
+    assert np.array_equal(layer.forward(x, logits)["y"], ref.forward(x, logits)["y"])
+    if hb == 3:                                                  # expert 1 is 3-bit already: mask has no effect on it
+        g0, u0, _ = layer.effective_weights(1)
+        layer.set_channel_switch([np.array([], np.int32)] * 4)
+        g1, u1, _ = layer.effective_weights(1)
+        assert np.array_equal(g0, g1) and np.array_equal(u0, u1)
+    layer.set_channel_precision([8] * 4, ug, uu)
+    layer.set_channel_switch([np.arange(0, layer.d, 3)] * 4)
+    assert np.array_equal(layer.forward(x, logits)["y"], y8)
 
 
 def test_empty_set_is_base_and_8bit_expert_ignores_mask():
