@@ -344,3 +344,6 @@ def select_significant(stats: np.ndarray, pool: np.ndarray, n_select: int, switc
         order = sorted(range(pool.shape[1]), key=lambda j: (-float(stats[e, j]), int(pool[e, j])))
         sets.append(np.array([pool[e, j] for j in order[: min(n_select, pool.shape[1])]], dtype=np.int32))
     return sets
+
+
+from . import assign  # noqa: E402,F401  (offline bit-width assignment, Algorithm 1)
