@@ -48,7 +48,8 @@ typedef enum {
     DYNAMO_ERR_STATE = 9,           /* call made before dynamo_pack_experts */
     DYNAMO_ERR_TOKENS = 10,         /* T < 0 or T > max_tokens */
     DYNAMO_ERR_CUDA = 11,           /* a CUDA runtime call failed */
-    DYNAMO_ERR_TIMEOUT = 12         /* a bounded device-side wait expired (see dynamo_poll_status) */
+    DYNAMO_ERR_TIMEOUT = 12,        /* a bounded device-side wait expired (see dynamo_poll_status) */
+    DYNAMO_ERR_ARG = 13             /* a scalar or array value is outside its domain (dynamo_assign_bits) */
 } dynamo_status;
 
 typedef struct {
@@ -223,6 +224,35 @@ dynamo_status dynamo_set_stats_collection(dynamo_ctx* ctx, int32_t on);
 dynamo_status dynamo_get_channel_stats(dynamo_ctx* ctx, float* stats_out, void* stream);
 dynamo_status dynamo_select_significant(dynamo_ctx* ctx, int32_t n_select, int32_t reset, int32_t* sig_idx_out,
                                         int32_t* sig_cnt_out, void* stream);
+
+/* Offline bit-width assignment (Section IV-A, Algorithm 1 and the two paragraphs around it): fuzzy c-means over the
+ * experts' significance, clusters mapped to precisions by significance, experts in the overlap of two clusters sent
+ * to the lower precision.  HOST code in double precision: every pointer is a host pointer, there is no context, no
+ * device work and no stream.  The result can be handed to dynamo_pack_experts (bits) or, after the significance was
+ * measured again on new data, to dynamo_set_channel_precision (Section IV-B: the difference between the two
+ * clusterings decides the precision the cached channels are requantized to).
+ *   x           : [n, dim] significance of each expert (the paper's x_i; dim = 1 there)
+ *   c           : number of clusters (the paper: 4), 1 <= c <= min(n, 16)
+ *   m, eps      : fuzzifier (> 1) and tolerance (>= 0) of Algorithm 1; the loop ends when the Frobenius norm of
+ *                 U_new - U_old is below eps, or after max_iter (>= 1) iterations
+ *   u0          : [n, c] initial memberships, every entry in [0, 1], every row summing to 1 (1e-9), or NULL
+ *   token_share : [n] each expert's share of the routed tokens, used when u0 is NULL: the initial memberships are
+ *                 those of the share against c anchors spread evenly from the smallest to the largest share
+ *                 (all equal, or c = 1: 1/c everywhere)
+ *   levels      : [c] precision of the most ... least significant cluster, each in {2, 3, 4, 6, 8}
+ *   overlap     : >= 0; an expert whose two largest memberships differ by less than this takes the lower of the two
+ *                 clusters' precisions (0: plain arg-max; exact ties always resolve to the lower precision)
+ * Each iteration: v_k = sum_i u_ik^m x_i / sum_i u_ik^m, then u_ik = 1 / sum_j (|x_i - v_k| / |x_i - v_j|)^(2/(m-1));
+ * a point lying on one or more centers shares its membership equally among them.  Clusters are ranked by the mean
+ * coordinate of their center (ties: larger membership mass, then lower index).
+ * Outputs: bits_out [n]; optional (NULL to skip) cluster_out [n], v_out [c, dim], u_out [n, c], iters_out [1].
+ * Errors (outputs untouched): NULL x / levels / bits_out, or u0 and token_share both NULL -> ERR_NULL; n, dim, c or
+ * max_iter out of range -> ERR_SHAPE; a level outside the list -> ERR_BITS; m <= 1, eps < 0, overlap < 0, a
+ * non-finite value, u0 not row-stochastic, or a cluster left without any membership -> ERR_ARG. */
+dynamo_status dynamo_assign_bits(const double* x, int32_t n, int32_t dim, int32_t c, double m, double eps,
+                                 int32_t max_iter, const double* u0, const double* token_share,
+                                 const int32_t* levels, double overlap, int32_t* bits_out, int32_t* cluster_out,
+                                 double* v_out, double* u_out, int32_t* iters_out);
 
 /* Which kernel serves small batches (forwards of at most 64 tokens, where every expert has few rows and the
  * forward is bound by streaming the packed weights of Section V-B from HBM):

@@ -28,12 +28,12 @@ DECODE_TENSOR, DECODE_STREAM = 0, 1
 PREFILL_PAIR, PREFILL_SINGLE = 0, 1
 
 STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_BITS", "ERR_ALIGN", "ERR_ARENA_TOO_SMALL", "ERR_INDEX_RANGE",
-                "ERR_INDEX_DUP", "ERR_NOT_CACHED", "ERR_STATE", "ERR_TOKENS", "ERR_CUDA", "ERR_TIMEOUT"]
+                "ERR_INDEX_DUP", "ERR_NOT_CACHED", "ERR_STATE", "ERR_TOKENS", "ERR_CUDA", "ERR_TIMEOUT", "ERR_ARG"]
 
 EXPORTED = ["dynamo_create", "dynamo_destroy", "dynamo_arena_bytes", "dynamo_pack_experts",
             "dynamo_set_channel_switch", "dynamo_set_channel_switch_many", "dynamo_set_switch_mode",
             "dynamo_moe_forward", "dynamo_moe_forward_router", "dynamo_moe_forward_host", "dynamo_export_codes", "dynamo_expert_stream_bytes",
-            "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_decode_kernel", "dynamo_set_prefill_kernel", "dynamo_set_stats_collection", "dynamo_set_channel_precision",
+            "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_decode_kernel", "dynamo_set_prefill_kernel", "dynamo_set_stats_collection", "dynamo_set_channel_precision", "dynamo_assign_bits",
             "dynamo_get_channel_stats", "dynamo_select_significant", "dynamo_route_permute_static", "dynamo_kernel_launches", "dynamo_status_str"]
 
 
@@ -83,6 +83,9 @@ def load():
         L.dynamo_set_prefill_kernel.argtypes = [vp, i32]
         L.dynamo_set_stats_collection.argtypes = [vp, i32]
         L.dynamo_set_channel_precision.argtypes = [vp, i32p, vp]
+        f64p = ctypes.POINTER(ctypes.c_double)
+        L.dynamo_assign_bits.argtypes = [f64p, i32, i32, i32, ctypes.c_double, ctypes.c_double, i32, f64p, f64p, i32p,
+                                         ctypes.c_double, i32p, i32p, f64p, f64p, i32p]
         L.dynamo_get_channel_stats.argtypes = [vp, vp, vp]
         L.dynamo_select_significant.argtypes = [vp, i32, i32, i32p, i32p, vp]
         L.dynamo_route_permute_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
@@ -395,3 +398,29 @@ def set_channel_switch_many(layers: List[DynamoLayer], sets_per_layer: Sequence[
     cnt = np.ascontiguousarray(np.stack(cnts), dtype=np.int32)
     st = dynamo_set_channel_switch_many([l.ctx for l in layers], idx, cnt, _stream())
     _check(st, "dynamo_set_channel_switch_many")
+
+
+def assign_bits(x, levels, c: int = 4, m: float = 2.0, eps: float = 1e-9, max_iter: int = 1000, u0=None,
+                token_share=None, overlap: float = 0.0):
+    """Offline bit-width assignment (Algorithm 1 + cluster-to-precision map).  Host arrays in, host arrays out:
+    returns dict(bits [n], cluster [n], V [c, dim], U [n, c], iters)."""
+    x = np.ascontiguousarray(np.asarray(x, dtype=np.float64))
+    if x.ndim == 1:
+        x = x[:, None]
+    n, dim = x.shape
+    f64p = ctypes.POINTER(ctypes.c_double)
+    as_f64 = lambda a: None if a is None else np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+    u0a, sha = as_f64(u0), as_f64(token_share)
+    if u0a is not None:
+        assert u0a.shape == (n, c)
+    if sha is not None:
+        assert sha.shape == (n,)
+    lv = np.ascontiguousarray(np.asarray(levels, dtype=np.int32))
+    assert lv.shape == (c,)
+    bits, cluster = np.zeros(n, np.int32), np.zeros(n, np.int32)
+    V, U, iters = np.zeros((c, dim)), np.zeros((n, c)), np.zeros(1, np.int32)
+    ptr = lambda a: None if a is None else a.ctypes.data_as(f64p)
+    st = load().dynamo_assign_bits(ptr(x), n, dim, c, m, eps, max_iter, ptr(u0a), ptr(sha), _i32p(lv), overlap,
+                                   _i32p(bits), _i32p(cluster), ptr(V), ptr(U), _i32p(iters))
+    _check(st, "dynamo_assign_bits")
+    return dict(bits=bits, cluster=cluster, V=V, U=U, iters=int(iters[0]))

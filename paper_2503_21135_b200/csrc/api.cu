@@ -275,6 +275,7 @@ const char* dynamo_status_str(dynamo_status s) {
         case DYNAMO_ERR_TOKENS: return "token count out of range";
         case DYNAMO_ERR_CUDA: return "CUDA runtime error";
         case DYNAMO_ERR_TIMEOUT: return "device-side wait expired";
+        case DYNAMO_ERR_ARG: return "argument value outside its domain";
     }
     return "unknown status";
 }

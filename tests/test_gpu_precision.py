@@ -137,3 +137,26 @@ def test_precision_errors_leave_state(lay):
     with pytest.raises(binding.DynamoError) as ei:
         fresh.set_channel_precision([8] * E)
     assert ei.value.status == binding.STATUS_NAMES.index("ERR_STATE")
+
+
+def test_recluster_on_new_data_sets_the_target_precision(lay):
+    # Section IV-B loop: expert loads measured on the data at hand -> Algorithm 1 -> per-expert target precision of the
+    # cached channels (higher or lower than before), on both sides
+    gpu, ora = lay["gpu"], lay["ora"]
+    E = CFG.n_experts
+    x, lg = wl.activations(CFG, 256, step=9), wl.router_logits(CFG, 256, step=9)
+    _, dbg = gpu.forward(x.cuda(), lg.cuda(), binding.F32, debug=True)
+    counts = np.diff(dbg["offsets"].cpu().numpy()).astype(np.float64)
+    assert counts.sum() == 256 * CFG.top_k
+    share = counts / counts.sum()
+    got = binding.assign_bits(share, [8, 6, 4, 3], token_share=share, overlap=0.05)
+    U0 = oracle.assign.initial_memberships(share.tolist(), 4, 2.0)
+    V, U, _, _ = oracle.assign.fuzzy_cmeans(share[:, None].tolist(), U0)
+    ref_bits, _ = oracle.assign.assign_bits(V, U, [8, 6, 4, 3], overlap=0.05)
+    assert got["bits"].tolist() == ref_bits and len(set(ref_bits)) >= 2
+    gpu.set_channel_precision(got["bits"])
+    ora.set_channel_precision(ref_bits, lay["ug"], lay["uu"])
+    _check_pool(lay)
+    _check_forward(lay, 64, step=10)
+    gpu.set_channel_precision([8] * E)
+    ora.set_channel_precision([8] * E, lay["ug"], lay["uu"])
