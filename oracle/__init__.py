@@ -69,7 +69,8 @@ def lib():
         L.orc_permute.restype = None
         L.orc_permute.argtypes = [i32p, i64, ci, ci, i32p, i32p]
         L.orc_expert_ffn.restype = None
-        L.orc_expert_ffn.argtypes = [u16p, i32p, i64, i64, i64, ci] + [u8p, u16p, u16p] * 5 + [u8p, f64p]
+        L.orc_expert_ffn.argtypes = ([u16p, i32p, i64, i64, i64, ci] + [u8p, u16p, u16p] * 5 + [u8p] +
+                                     [u8p, u16p, u16p] + [u8p, f64p])
         L.orc_threads.restype = ci
         L.orc_set_threads.argtypes = [ci]
         _lib = L
@@ -207,7 +208,9 @@ class OracleLayer:
     ``w_gate``/``w_up``: uint16 (bf16 bits) [E+Es, f, d]; ``w_down``: [E+Es, d, f].
     ``bits``: base bit-width per expert.  The 8-bit ("hi") quantization of W_gate and
     W_up is kept for every routed expert with base bits < 8: a significant channel takes
-    the value it has in that uniform 8-bit quantization.
+    the value it has in that uniform 8-bit quantization.  The same holds on the d_ff side
+    (``set_channel_switch_down``): a significant INPUT channel c of W_down, c in [0, f),
+    takes column c of the uniform 8-bit quantization of W_down.
     """
 
     def __init__(self, w_gate, w_up, w_down, bits: Sequence[int], G: int, n_experts: int, top_k: int,
@@ -226,6 +229,28 @@ class OracleLayer:
             if e < self.E and b < HI_BITS:
                 self.hi[e] = tuple(QuantMatrix(*quantize(w[e], G, HI_BITS)) for w in (w_gate, w_up))
         self.sig: List[np.ndarray] = [np.zeros((0,), np.int32) for _ in range(self.E)]
+        self.hi_down: List[Optional[QuantMatrix]] = [None] * self.n_total
+        self.sig_down: List[np.ndarray] = [np.zeros((0,), np.int32) for _ in range(self.E)]
+
+    def enable_down_side(self, w_down) -> None:
+        """Keep the uniform 8-bit quantization of W_down for every routed expert with base bits < 8
+        (Section IV-B applied to the channels of the second projection: its input channels are the d_ff
+        hidden units).  w_down: the original bf16 bit patterns [E+Es, d, f]."""
+        for e in range(self.E):
+            if self.base[e] is not None and self.bits[e] < HI_BITS:
+                self.hi_down[e] = QuantMatrix(*quantize(w_down[e], self.G, HI_BITS))
+
+    def set_channel_switch_down(self, sets: Sequence[np.ndarray]) -> None:
+        """Install the significant set of W_down's input channels (indices in [0, f)) of every routed expert."""
+        assert len(sets) == self.E
+        self.sig_down = [np.unique(np.asarray(s, dtype=np.int32)) for s in sets]
+
+    def mask_down(self, e: int) -> Optional[np.ndarray]:
+        if e >= self.E or self.hi_down[e] is None or len(self.sig_down[e]) == 0:
+            return None
+        mk = np.zeros((self.f,), np.uint8)
+        mk[self.sig_down[e]] = 1
+        return mk
 
     def set_channel_precision(self, hi_bits: Sequence[int], w_gate, w_up) -> None:
         """Precision the significant channels are served at, per routed expert (Section IV-B: the replaced
@@ -258,6 +283,11 @@ class OracleLayer:
             g8, u8 = (dequantize(qm.q, qm.s, qm.m, self.G) for qm in self.hi[e])
             g[:, cols] = g8[:, cols]
             u[:, cols] = u8[:, cols]
+        mkd = self.mask_down(e)
+        if mkd is not None:
+            cols = np.nonzero(mkd)[0]
+            qm = self.hi_down[e]
+            dn[:, cols] = dequantize(qm.q, qm.s, qm.m, self.G)[:, cols]
         return g, u, dn
 
     def expert_ffn(self, x_u16: np.ndarray, e: int, rows: np.ndarray) -> np.ndarray:
@@ -275,8 +305,14 @@ class OracleLayer:
                 args += [_p(qm.q, u8), _p(qm.s, u16), _p(qm.m, u16)]
         else:
             args += [_p(None, u8), _p(None, u16), _p(None, u16)] * 2
+        mkd = self.mask_down(e)
+        if mkd is not None:
+            qm = self.hi_down[e]
+            dargs = [_p(qm.q, u8), _p(qm.s, u16), _p(qm.m, u16), _p(mkd, u8)]
+        else:
+            dargs = [_p(None, u8), _p(None, u16), _p(None, u16), _p(None, u8)]
         lib().orc_expert_ffn(_p(np.ascontiguousarray(x_u16), u16), _p(rows, ctypes.c_int32), len(rows),
-                             self.d, self.f, self.G, *args, _p(mk, u8), _p(out, ctypes.c_double))
+                             self.d, self.f, self.G, *args, _p(mk, u8), *dargs, _p(out, ctypes.c_double))
         return out
 
     def forward(self, x_u16: np.ndarray, logits: np.ndarray, tokens: Optional[np.ndarray] = None):

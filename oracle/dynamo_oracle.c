@@ -213,7 +213,8 @@ void orc_permute(const int32_t* idx, int64_t T, int k, int E, int32_t* offsets, 
 /* ---- C5 + C6: one expert's SwiGLU FFN over effective weights ------------------------------
  * Effective weight (Sections IV-B, V-A: significant channels are served from the channel cache
  * at the higher precision, the rest at the expert's base precision):
- *   W_eff[n, c] = s8[n, c/G]*q8[n, c] + m8[n, c/G]   if mask != NULL and mask[c]   (gate, up only)
+ *   W_eff[n, c] = s8[n, c/G]*q8[n, c] + m8[n, c/G]   if mask != NULL and mask[c]   (gate, up: c an input channel
+ *                                                       in [0, d); down: mask_d over its input channels [0, f))
  *               = sb[n, c/G]*qb[n, c] + mb[n, c/G]   otherwise.
  * FFN:  g = W_gate,eff x,  u = W_up,eff x,  h = g / (1 + exp(-g)) * u,  y = W_down h,
  * all in double with no intermediate rounding.  x rows are bf16 bit patterns [T, d];
@@ -224,7 +225,9 @@ void orc_expert_ffn(const uint16_t* x, const int32_t* rows, int64_t n_rows, int6
                     const uint8_t* qd, const uint16_t* sd, const uint16_t* md,
                     const uint8_t* q8g, const uint16_t* s8g, const uint16_t* m8g,
                     const uint8_t* q8u, const uint16_t* s8u, const uint16_t* m8u,
-                    const uint8_t* mask, double* out) {
+                    const uint8_t* mask,
+                    const uint8_t* q8d, const uint16_t* s8d, const uint16_t* m8d, const uint8_t* mask_d,
+                    double* out) {
     double* h = (double*)malloc(sizeof(double) * (size_t)(n_rows * f > 0 ? n_rows * f : 1));
     double* xd = (double*)malloc(sizeof(double) * (size_t)(n_rows * d > 0 ? n_rows * d : 1));
     for (int64_t i = 0; i < n_rows; ++i)
@@ -256,7 +259,8 @@ void orc_expert_ffn(const uint16_t* x, const int32_t* rows, int64_t n_rows, int6
         double* wd = (double*)malloc(sizeof(double) * (size_t)f);
 #pragma omp for schedule(static)
         for (int64_t n = 0; n < d; ++n) {
-            for (int64_t c = 0; c < f; ++c) wd[c] = deq(qd, sd, md, n, c, f, G);
+            for (int64_t c = 0; c < f; ++c)
+                wd[c] = (mask_d && mask_d[c]) ? deq(q8d, s8d, m8d, n, c, f, G) : deq(qd, sd, md, n, c, f, G);
             for (int64_t i = 0; i < n_rows; ++i) {
                 double y = 0.0;
                 const double* hr = h + i * f;

@@ -253,6 +253,10 @@ def _numpy_eff(layer, e):
             h = layer.hi[e][i]
             w8 = np.repeat(f16_to_f64(h.s), G, axis=1) * h.q + np.repeat(f16_to_f64(h.m), G, axis=1)
             w[:, layer.sig[e]] = w8[:, layer.sig[e]]
+        if i == 2 and e < layer.E and layer.hi_down[e] is not None and len(layer.sig_down[e]):
+            h = layer.hi_down[e]
+            w8 = np.repeat(f16_to_f64(h.s), G, axis=1) * h.q + np.repeat(f16_to_f64(h.m), G, axis=1)
+            w[:, layer.sig_down[e]] = w8[:, layer.sig_down[e]]
         mats.append(w)
     return mats
 
@@ -358,6 +362,37 @@ def test_channel_precision_all_switched_equals_uniform_target(hb):
     layer.set_channel_precision([8] * 4, ug, uu)
     layer.set_channel_switch([np.arange(0, layer.d, 3)] * 4)
     assert np.array_equal(layer.forward(x, logits)["y"], y8)
+
+
+def test_down_side_set_brute_force_and_identities():
+    # significant INPUT channels of W_down (indices in [0, f)): the forward equals the token-major brute force on
+    # independently rebuilt effective weights; all channels switched on both sides = the uniform 8-bit layer;
+    # the empty set is the base; the 8-bit expert ignores its set
+    layer, x, logits, (wg, wu, wd) = _tiny_layer(seed=12, bits=(2, 3, 4, 8))
+    base = layer.forward(x, logits)["y"]
+    layer.enable_down_side(bf16_bits(wd))
+    assert layer.hi_down[3] is None and layer.hi_down[0] is not None
+    assert np.array_equal(layer.forward(x, logits)["y"], base)
+    layer.set_channel_switch([np.array([3, 7, 64]), np.array([], np.int32), np.array([3]), np.array([1])])
+    layer.set_channel_switch_down([np.array([0, 5, 191]), np.array([64, 65]), np.array([], np.int32), np.array([2, 9])])
+    out = layer.forward(x, logits)["y"]
+    ref = _dense_token_major(layer, x, logits)
+    assert np.max(np.abs(out - ref)) <= 1e-12 * np.max(np.abs(ref))
+    assert not np.array_equal(out, base)
+    for e in range(4):
+        for a, b in zip(layer.effective_weights(e), _numpy_eff(layer, e)):
+            assert np.array_equal(a, b)
+    _, _, d0 = layer.effective_weights(0)
+    changed = np.nonzero(np.any(d0 != oracle.dequantize(*[getattr(layer.base[0][2], k) for k in "qsm"], layer.G), axis=0))[0]
+    assert set(changed.tolist()) <= {0, 5, 191} and len(changed) >= 2       # only the listed columns move
+    # everything switched on both sides == uniform 8-bit layer
+    ref8 = oracle.OracleLayer(bf16_bits(wg), bf16_bits(wu), bf16_bits(wd), [8, 8, 8, 8], layer.G, 4, 2)
+    layer.set_channel_switch([np.arange(layer.d)] * 4)
+    layer.set_channel_switch_down([np.arange(layer.f)] * 4)
+    assert np.array_equal(layer.forward(x, logits)["y"], ref8.forward(x, logits)["y"])
+    layer.set_channel_switch([np.array([], np.int32)] * 4)
+    layer.set_channel_switch_down([np.array([], np.int32)] * 4)
+    assert np.array_equal(layer.forward(x, logits)["y"], base)
 
 
 def test_empty_set_is_base_and_8bit_expert_ignores_mask():
