@@ -98,7 +98,8 @@ class ClockSampler:
         return out
 
 
-def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None, decode_kernel=None, prefill_kernel=None):
+def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None, decode_kernel=None, prefill_kernel=None,
+                 down_side=0):
     """Generate, upload and pack ``n_layers`` independent layers; they share one workspace."""
     from paper_2503_21135_b200 import binding
 
@@ -111,6 +112,10 @@ def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None, decode_ker
         layer = binding.DynamoLayer.from_config(cfg, max_tokens=max_tokens, workspace=ws, device=device)
         layer.pack_experts(wg.to(device), wu.to(device), wd.to(device), bits, pool)
         layer.set_channel_switch(sets)
+        if down_side > 0:  # significant hidden units on the d_ff side: 2 * down_side cached, down_side significant
+            pool_d = wl.cache_pool_down(cfg, 2 * down_side, l)
+            layer.pack_down_cache(wd.to(device), bits, pool_d, down_side)
+            layer.set_channel_switch_down(wl.sig_sets_down(cfg, pool_d, down_side, l))
         if tc_min_rows is not None:
             layer.set_tc_min_rows(tc_min_rows)
         if prefill_kernel is not None:
@@ -197,7 +202,8 @@ def run_ours(args, rank, world, device):
         if world > 1:
             torch.distributed.barrier()
 
-    layers, meta = build_layers(cfg, n_layers, max(T, max(cfg.tokens)), device, args.tc_min_rows, args.decode_kernel, args.prefill_kernel)
+    layers, meta = build_layers(cfg, n_layers, max(T, max(cfg.tokens)), device, args.tc_min_rows, args.decode_kernel, args.prefill_kernel,
+                                args.down_side)
     sweep_T = sorted(set([T] + (list(cfg.tokens) if args.sweep else [])))
     results = {}
     for Tcur in sweep_T:
@@ -288,7 +294,8 @@ def run_ours(args, rank, world, device):
         "config": {"workload": f"{cfg.name}: d_model={cfg.d_model} d_ff={cfg.d_ff} E={cfg.n_experts} top{cfg.top_k} "
                                f"G={cfg.group_size} S={cfg.max_sig} T={T}",
                    "tokens": T, "layers_rotated": n_layers, "l2": "inputs larger than L2 (rotating layer arenas)",
-                   "parallelism": "replicas only" if world > 1 else "single gpu"},
+                   "parallelism": "replicas only" if world > 1 else "single gpu",
+                   **({"down_side_significant": args.down_side} if args.down_side else {})},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": T * cfg.d_model * 2 + T * cfg.n_experts * 4,
                 "d2h_bytes_per_step": T * cfg.d_model * 4},
         "gpu_launches": r["launches"],
@@ -493,6 +500,8 @@ def main():
                     help="kernel for batches of up to 64 tokens (default: the library's, stream)")
     ap.add_argument("--router", action="store_true",
                     help="also time the forward with the router GEMM + top-k fused in front")
+    ap.add_argument("--down-side", type=int, default=0,
+                    help="also serve this many significant hidden units per expert at 8-bit on the d_ff side (W_down)")
     ap.add_argument("--sweep", action="store_true", help="also time the workload's other token counts")
     ap.add_argument("--cpu-tokens", type=int, default=16, help="tokens in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -225,6 +225,39 @@ dynamo_status dynamo_get_channel_stats(dynamo_ctx* ctx, float* stats_out, void* 
 dynamo_status dynamo_select_significant(dynamo_ctx* ctx, int32_t n_select, int32_t reset, int32_t* sig_idx_out,
                                         int32_t* sig_cnt_out, void* stream);
 
+/* Significant channels on the d_ff side (Section IV-B applied to the second projection: the input channels of
+ * W_down are the hidden units).  Optional; a layer that never calls these pays nothing.
+ * A significant hidden unit c of routed expert e (base bits < 8) takes column c of the expert's uniform 8-bit
+ * quantization of W_down (same groups of G hidden units, same quantizer as dynamo_pack_experts).  The forward
+ * realises it as the base down GEMM plus, between that GEMM and the combine, one kernel that adds
+ * h[row][c] * (W8[n][c] - Wbase[n][c]) over the significant c, the difference kept as fp16 per (cached channel, n).
+ *
+ * dynamo_down_cache_bytes: size of the caller-owned arena (256-byte aligned device memory that must outlive the
+ *   context's use of it) for cache_size_down cached hidden units per expert and sets of up to max_sig_down.
+ * dynamo_pack_down_cache: after dynamo_pack_experts (a new dynamo_pack_experts drops the cache).
+ *   w_down         : device bf16 [E + E_s, d_model, d_ff], the originals given to dynamo_pack_experts
+ *   cache_idx_down : host int32 [E, cache_size_down], strictly increasing per expert, each in [0, d_ff)
+ *   Builds the 8-bit parameters of every (row, group) of W_down and, per cached hidden unit, its 8-bit codes, bf16
+ *   originals (the channel cache) and differences.  All sets start empty.  Synchronises the stream.
+ * dynamo_set_channel_switch_down: installs the sets (the state depends only on the last call).
+ *   sig_idx : host int32 [E, max_sig_down], sig_cnt : host int32 [E], 0 <= cnt <= max_sig_down
+ *   8-bit experts are validated but keep the empty set.  Synchronises the stream.
+ * dynamo_export_codes with DYNAMO_MAT_DOWN and DYNAMO_CODES_HI_POOL / HI_ACTIVE returns the 8-bit codes of the
+ * cached / significant hidden units (0 elsewhere) and the 8-bit parameters, shaped like the base export.
+ * dynamo_set_channel_precision does not reach this side: it stays at 8 bits.
+ * Errors: NULL -> ERR_NULL; before dynamo_pack_experts (or, for the switch and the export, before
+ * dynamo_pack_down_cache) -> ERR_STATE; cache_size_down outside [1, min(d_ff, 65535)], max_sig_down outside
+ * [0, min(256, cache_size_down)] -> ERR_SHAPE; arena misaligned -> ERR_ALIGN, too small -> ERR_ARENA_TOO_SMALL; an
+ * index outside [0, d_ff) or a count outside its range -> ERR_INDEX_RANGE; a repeated or unsorted index ->
+ * ERR_INDEX_DUP; a significant unit that is not cached -> ERR_NOT_CACHED.  On an error the previous state stays. */
+dynamo_status dynamo_down_cache_bytes(const dynamo_layer_desc* desc, const int32_t* bits, int32_t cache_size_down,
+                                      int32_t max_sig_down, size_t* bytes);
+dynamo_status dynamo_pack_down_cache(dynamo_ctx* ctx, const void* w_down, const int32_t* cache_idx_down,
+                                     int32_t cache_size_down, int32_t max_sig_down, void* down_arena, size_t down_bytes,
+                                     void* stream);
+dynamo_status dynamo_set_channel_switch_down(dynamo_ctx* ctx, const int32_t* sig_idx, const int32_t* sig_cnt,
+                                             void* stream);
+
 /* Offline bit-width assignment (Section IV-A, Algorithm 1 and the two paragraphs around it): fuzzy c-means over the
  * experts' significance, clusters mapped to precisions by significance, experts in the overlap of two clusters sent
  * to the lower precision.  HOST code in double precision: every pointer is a host pointer, there is no context, no

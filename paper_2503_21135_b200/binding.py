@@ -34,6 +34,7 @@ EXPORTED = ["dynamo_create", "dynamo_destroy", "dynamo_arena_bytes", "dynamo_pac
             "dynamo_set_channel_switch", "dynamo_set_channel_switch_many", "dynamo_set_switch_mode",
             "dynamo_moe_forward", "dynamo_moe_forward_router", "dynamo_moe_forward_host", "dynamo_export_codes", "dynamo_expert_stream_bytes",
             "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_decode_kernel", "dynamo_set_prefill_kernel", "dynamo_set_stats_collection", "dynamo_set_channel_precision", "dynamo_assign_bits",
+            "dynamo_down_cache_bytes", "dynamo_pack_down_cache", "dynamo_set_channel_switch_down",
             "dynamo_get_channel_stats", "dynamo_select_significant", "dynamo_route_permute_static", "dynamo_kernel_launches", "dynamo_status_str"]
 
 
@@ -83,6 +84,9 @@ def load():
         L.dynamo_set_prefill_kernel.argtypes = [vp, i32]
         L.dynamo_set_stats_collection.argtypes = [vp, i32]
         L.dynamo_set_channel_precision.argtypes = [vp, i32p, vp]
+        L.dynamo_down_cache_bytes.argtypes = [vp, i32p, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
+        L.dynamo_pack_down_cache.argtypes = [vp, vp, i32p, i32, i32, vp, ctypes.c_size_t, vp]
+        L.dynamo_set_channel_switch_down.argtypes = [vp, i32p, i32p, vp]
         f64p = ctypes.POINTER(ctypes.c_double)
         L.dynamo_assign_bits.argtypes = [f64p, i32, i32, i32, ctypes.c_double, ctypes.c_double, i32, f64p, f64p, i32p,
                                          ctypes.c_double, i32p, i32p, f64p, f64p, i32p]
@@ -274,6 +278,35 @@ class DynamoLayer:
         idx, cnt = self.sig_arrays(sets)
         st = dynamo_set_channel_switch(self.ctx, np.ascontiguousarray(idx), cnt, _stream())
         _check(st, "dynamo_set_channel_switch")
+
+    def pack_down_cache(self, w_down: torch.Tensor, bits, cache_idx_down, max_sig_down: int):
+        """Channel cache on the d_ff side: cache_idx_down int [E, P2] (sorted hidden-unit indices per expert)."""
+        bits = np.ascontiguousarray(bits, dtype=np.int32)
+        ci = np.ascontiguousarray(cache_idx_down, dtype=np.int32)
+        assert ci.ndim == 2 and ci.shape[0] == self.desc.n_experts
+        assert w_down.is_cuda and w_down.dtype == torch.bfloat16 and w_down.is_contiguous()
+        P2 = int(ci.shape[1])
+        nbytes = ctypes.c_size_t(0)
+        _check(load().dynamo_down_cache_bytes(ctypes.byref(self.desc), _i32p(bits), P2, int(max_sig_down),
+                                              ctypes.byref(nbytes)), "dynamo_down_cache_bytes")
+        arena = torch.empty(nbytes.value, dtype=torch.uint8, device=self.device)
+        st = load().dynamo_pack_down_cache(self.ctx, w_down.data_ptr(), _i32p(ci), P2, int(max_sig_down),
+                                           arena.data_ptr(), arena.numel(), _stream())
+        _check(st, "dynamo_pack_down_cache")
+        self.down_arena = arena                  # on an error the previous arena stays referenced (and in use)
+        self.max_sig_down = int(max_sig_down)
+
+    def set_channel_switch_down(self, sets: Sequence[np.ndarray]):
+        E, S2 = self.desc.n_experts, self.max_sig_down
+        idx = np.full((E, max(S2, 1)), -1, dtype=np.int32)
+        cnt = np.zeros((E,), dtype=np.int32)
+        for e, s_ in enumerate(sets):
+            s_ = np.asarray(s_, dtype=np.int32)
+            cnt[e] = len(s_)
+            idx[e, : min(len(s_), S2)] = s_[:S2]
+        idx = np.ascontiguousarray(idx[:, :S2] if S2 > 0 else idx[:, :1])
+        st = load().dynamo_set_channel_switch_down(self.ctx, _i32p(idx), _i32p(cnt), _stream())
+        _check(st, "dynamo_set_channel_switch_down")
 
     def set_switch_mode(self, mode: int):
         _check(dynamo_set_switch_mode(self.ctx, mode), "dynamo_set_switch_mode")

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdynamo.so")
-SOURCES = ["api.cu", "pack.cu", "route.cu", "switch.cu", "stats.cu", "ffn_stream.cu", "ffn_tc.cu", "ffn_tc2.cu", "ffn_tcd.cu", "noalloc.cu", "assign.cu"]
+SOURCES = ["api.cu", "pack.cu", "route.cu", "switch.cu", "stats.cu", "ffn_stream.cu", "ffn_tc.cu", "ffn_tc2.cu", "ffn_tcd.cu", "noalloc.cu", "assign.cu", "downside.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "static"]
 

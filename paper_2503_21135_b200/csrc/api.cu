@@ -14,6 +14,11 @@ cudaError_t launch_pack_hi(const void* w_gate, const void* w_up, int f, int d, i
                            const int32_t* cache_idx_dev, const ExpertDev& ex, cudaStream_t st);
 cudaError_t launch_requant(const LayerDev* L, int f, const int32_t* items_dev, int n_items, cudaStream_t st);
 cudaError_t launch_retarget(LayerDev* L, int e, int f, int bits, cudaStream_t st);
+cudaError_t launch_pack_down_hi(const void* w_down, int d, int f, int G, int P2, const int32_t* cache_idx_dev,
+                                int base_bits, const DownExpertDev& ex, cudaStream_t st);
+cudaError_t launch_down_fix(const LayerDev* L, const DownDev* D2, const WsDev& ws, int d, cudaStream_t st);
+cudaError_t launch_export_down(const LayerDev* L, const DownDev* D2, int e, int which, long long n_elems, uint8_t* q,
+                               uint16_t* sc, uint16_t* zr, cudaStream_t st);
 cudaError_t launch_export(const LayerDev* L, int e, int mat, int which, long long n_elems, uint8_t* q, uint16_t* sc,
                           uint16_t* zr, cudaStream_t st);
 cudaError_t launch_route(const float* logits, int T, int E, int k, int renorm, int32_t* idx, float* w,
@@ -72,6 +77,38 @@ inline int ksplit_for(const dynamo_layer_desc& D, int T) {
     return R <= DECODE_ROWS ? std::min(MAX_KSPLIT, D.d_ff / KC) : 1;
 }
 inline int switch_ints_per_layer(const dynamo_layer_desc& D) { return D.n_experts * (2 * s_pad_of(D) + 1); }
+
+// Arena of the d_ff-side channel cache: header, tables, then per switchable expert the 8-bit parameters of W_down,
+// the cached channels' codes, differences and bf16 originals.
+struct DownLayout {
+    size_t cache_idx = 0, sig_chan = 0, sig_pool = 0, sig_cnt = 0;
+    std::vector<size_t> s8m8, q8, delta, cache_w;
+    size_t total = 0;
+};
+
+void down_layout(const dynamo_layer_desc& D, const int32_t* bits, int P2, int S2, DownLayout& A) {
+    const size_t d = D.d_model, f = D.d_ff, G = D.group_size, E = D.n_experts;
+    size_t off = align_up(sizeof(DownDev));
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    A.cache_idx = take(E * P2 * 4);
+    A.sig_chan = take(E * (size_t)std::max(S2, 1) * 4);
+    A.sig_pool = take(E * (size_t)std::max(S2, 1) * 4);
+    A.sig_cnt = take(E * 4);
+    A.s8m8.assign(E, 0); A.q8.assign(E, 0); A.delta.assign(E, 0); A.cache_w.assign(E, 0);
+    for (size_t e = 0; e < E; ++e) {
+        if (bits[e] >= HI_BITS) continue;
+        A.s8m8[e] = take(d * (f / G) * 4);
+        A.q8[e] = take((size_t)P2 * d);
+        A.delta[e] = take((size_t)P2 * d * 2);
+        A.cache_w[e] = take((size_t)P2 * d * 2);
+    }
+    A.total = off;
+}
+
+dynamo_status check_down_sizes(const dynamo_layer_desc& D, int P2, int S2) {
+    if (P2 < 1 || P2 > D.d_ff || P2 > 65535 || S2 < 0 || S2 > 256 || S2 > P2) return DYNAMO_ERR_SHAPE;
+    return DYNAMO_OK;
+}
 
 dynamo_status check_desc(const dynamo_layer_desc* D) {
     if (!D) return DYNAMO_ERR_NULL;
@@ -175,6 +212,13 @@ struct dynamo_ctx {
     bool packed = false;
     std::vector<int32_t> bits;
     std::vector<int32_t> hi_bits;                // precision the significant channels of each routed expert are served at
+    // d_ff-side channel cache (optional, its own caller-owned arena)
+    uint8_t* down_arena = nullptr;
+    int P2 = 0, S2 = 0;
+    DownLayout DA;
+    std::vector<int32_t> cache_idx_down;         // host copy [E][P2]
+    std::vector<std::vector<int32_t>> sig_down;  // current sets, in slot order
+    int down_active = 0;                         // experts whose d_ff-side set is not empty
     std::vector<int32_t> cache_idx;              // host copy [E][P]
     std::vector<std::vector<int32_t>> sig;       // current sets, in slot order
     ArenaLayout A;
@@ -446,6 +490,8 @@ dynamo_status dynamo_pack_experts(dynamo_ctx* ctx, const void* w_gate, const voi
     ctx->ws = (uint8_t*)workspace;
     ctx->bits.assign(bits, bits + n);
     ctx->hi_bits.assign(D.n_experts, HI_BITS);
+    ctx->down_arena = nullptr;  // a d_ff-side cache belongs to the previous packing
+    ctx->down_active = 0;
     ctx->cache_idx.assign(cache_idx, cache_idx + (size_t)D.n_experts * P);
     ctx->sig.assign(D.n_experts, {});
 
@@ -647,6 +693,10 @@ static dynamo_status forward_impl(dynamo_ctx* ctx, const void* x, const float* r
         if (ctx->prof_ev[1]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[1], st));
         CUDA_TRY(launch_ffn_tcd(L, ws, 0, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, ctx->n_sms, st));
         if (ctx->prof_ev[2]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[2], st));
+        if (ctx->down_active) {
+            CUDA_TRY(launch_down_fix(L, (const DownDev*)ctx->down_arena, ws, D.d_model, st));
+            ctx->launches += 1;
+        }
         CUDA_TRY(launch_combine(ws, D.d_model, D.top_k, D.n_shared, y, y_dtype == DYNAMO_F32, split_stride, st));
         ctx->launches += 6;
         return forward_debug_copies(ctx, ws, T, dbg, st);
@@ -662,6 +712,10 @@ static dynamo_status forward_impl(dynamo_ctx* ctx, const void* x, const float* r
     if (use_tc) CUDA_TRY(pair ? launch_ffn_tc2(L, ws, 0, ctx->host_layer.n_rb2, n, ctx->n_sms, st)
                               : launch_ffn_tc(L, ws, 0, ctx->host_layer.n_rb2, n, ctx->n_sms, st));
     if (ctx->prof_ev[2]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[2], st));
+    if (ctx->down_active) {  // significant hidden units: add what their 8-bit columns of W_down change
+        CUDA_TRY(launch_down_fix(L, (const DownDev*)ctx->down_arena, ws, D.d_model, st));
+        ctx->launches += 1;
+    }
     CUDA_TRY(launch_combine(ws, D.d_model, D.top_k, D.n_shared, y, y_dtype == DYNAMO_F32, split_stride, st));
     ctx->launches += use_tc ? 8 : 6;
     return forward_debug_copies(ctx, ws, T, dbg, st);
@@ -703,6 +757,123 @@ dynamo_status dynamo_moe_forward_host(dynamo_ctx* ctx, const void* x_host, const
     return DYNAMO_OK;
 }
 
+dynamo_status dynamo_down_cache_bytes(const dynamo_layer_desc* desc, const int32_t* bits, int32_t cache_size_down,
+                                      int32_t max_sig_down, size_t* bytes) {
+    if (!bytes) return DYNAMO_ERR_NULL;
+    dynamo_status s = check_desc(desc);
+    if (s != DYNAMO_OK) return s;
+    s = check_bits(*desc, bits);
+    if (s != DYNAMO_OK) return s;
+    s = check_down_sizes(*desc, cache_size_down, max_sig_down);
+    if (s != DYNAMO_OK) return s;
+    DownLayout A;
+    down_layout(*desc, bits, cache_size_down, max_sig_down, A);
+    *bytes = A.total;
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_pack_down_cache(dynamo_ctx* ctx, const void* w_down, const int32_t* cache_idx_down,
+                                     int32_t cache_size_down, int32_t max_sig_down, void* down_arena, size_t down_bytes,
+                                     void* stream) {
+    if (!ctx || !w_down || !cache_idx_down || !down_arena) return DYNAMO_ERR_NULL;
+    if (!ctx->packed) return DYNAMO_ERR_STATE;
+    const dynamo_layer_desc& D = ctx->D;
+    dynamo_status s = check_down_sizes(D, cache_size_down, max_sig_down);
+    if (s != DYNAMO_OK) return s;
+    if ((uintptr_t)down_arena % ALIGN) return DYNAMO_ERR_ALIGN;
+    const int P2 = cache_size_down, S2 = max_sig_down, E = D.n_experts;
+    DownLayout A;
+    down_layout(D, ctx->bits.data(), P2, S2, A);
+    if (down_bytes < A.total) return DYNAMO_ERR_ARENA_TOO_SMALL;
+    for (int e = 0; e < E; ++e)
+        for (int j = 0; j < P2; ++j) {
+            const int c = cache_idx_down[(size_t)e * P2 + j];
+            if (c < 0 || c >= D.d_ff) return DYNAMO_ERR_INDEX_RANGE;
+            if (j > 0 && c <= cache_idx_down[(size_t)e * P2 + j - 1]) return DYNAMO_ERR_INDEX_DUP;
+        }
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t* base = (uint8_t*)down_arena;
+    ctx->down_arena = nullptr;  // stays off if anything below fails
+    ctx->down_active = 0;
+    ctx->P2 = P2;
+    ctx->S2 = S2;
+    ctx->DA = A;
+    ctx->cache_idx_down.assign(cache_idx_down, cache_idx_down + (size_t)E * P2);
+    ctx->sig_down.assign(E, {});
+
+    std::vector<uint8_t> hdr(sizeof(DownDev), 0);
+    DownDev& H = *reinterpret_cast<DownDev*>(hdr.data());
+    H.P2 = P2;
+    H.S2 = std::max(S2, 1);
+    H.cache_idx = (int32_t*)(base + A.cache_idx);
+    H.sig_chan = (int32_t*)(base + A.sig_chan);
+    H.sig_pool = (int32_t*)(base + A.sig_pool);
+    H.sig_cnt = (int32_t*)(base + A.sig_cnt);
+    for (int e = 0; e < E; ++e) {
+        if (ctx->bits[e] >= HI_BITS) continue;
+        H.ex[e].s8m8 = (uint32_t*)(base + A.s8m8[e]);
+        H.ex[e].q8 = base + A.q8[e];
+        H.ex[e].delta = (__half*)(base + A.delta[e]);
+        H.ex[e].cache_w = (__nv_bfloat16*)(base + A.cache_w[e]);
+    }
+    CUDA_TRY(cudaMemcpyAsync(base, hdr.data(), sizeof(DownDev), cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(H.cache_idx, ctx->cache_idx_down.data(), (size_t)E * P2 * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemsetAsync(H.sig_chan, 0xff, (size_t)E * H.S2 * 4, st));
+    CUDA_TRY(cudaMemsetAsync(H.sig_pool, 0, (size_t)E * H.S2 * 4, st));
+    CUDA_TRY(cudaMemsetAsync(H.sig_cnt, 0, (size_t)E * 4, st));
+    const char* wd = (const char*)w_down;
+    const size_t per_expert = (size_t)D.d_model * D.d_ff * 2;
+    for (int e = 0; e < E; ++e) {
+        if (ctx->bits[e] >= HI_BITS) continue;
+        CUDA_TRY(launch_pack_down_hi(wd + e * per_expert, D.d_model, D.d_ff, D.group_size, P2,
+                                     H.cache_idx + (size_t)e * P2, ctx->bits[e], H.ex[e], st));
+        ctx->launches += 1;
+    }
+    CUDA_TRY(cudaStreamSynchronize(st));  // the host staging above may go away
+    ctx->down_arena = base;
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_set_channel_switch_down(dynamo_ctx* ctx, const int32_t* sig_idx, const int32_t* sig_cnt,
+                                             void* stream) {
+    if (!ctx || !sig_idx || !sig_cnt) return DYNAMO_ERR_NULL;
+    if (!ctx->packed || !ctx->down_arena) return DYNAMO_ERR_STATE;
+    const dynamo_layer_desc& D = ctx->D;
+    const int E = D.n_experts, P2 = ctx->P2, S2 = ctx->S2, S2d = std::max(S2, 1);
+    std::vector<int32_t> chan((size_t)E * S2d, -1), pool((size_t)E * S2d, 0), cnts(E, 0);
+    std::vector<std::vector<int32_t>> lists(E);
+    std::vector<uint8_t> seen(D.d_ff);
+    for (int e = 0; e < E; ++e) {
+        const int cnt = sig_cnt[e];
+        if (cnt < 0 || cnt > S2) return DYNAMO_ERR_INDEX_RANGE;
+        std::fill(seen.begin(), seen.end(), 0);
+        const int32_t* ci = ctx->cache_idx_down.data() + (size_t)e * P2;
+        for (int j = 0; j < cnt; ++j) {
+            const int ch = sig_idx[(size_t)e * S2 + j];
+            if (ch < 0 || ch >= D.d_ff) return DYNAMO_ERR_INDEX_RANGE;
+            if (seen[ch]) return DYNAMO_ERR_INDEX_DUP;
+            seen[ch] = 1;
+            const int32_t* it = std::lower_bound(ci, ci + P2, ch);
+            if (it == ci + P2 || *it != ch) return DYNAMO_ERR_NOT_CACHED;
+            if (ctx->bits[e] >= HI_BITS) continue;  // an 8-bit expert ignores its set
+            chan[(size_t)e * S2d + lists[e].size()] = ch;
+            pool[(size_t)e * S2d + lists[e].size()] = (int32_t)(it - ci);
+            lists[e].push_back(ch);
+        }
+        cnts[e] = (int32_t)lists[e].size();
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t* base = ctx->down_arena;
+    CUDA_TRY(cudaMemcpyAsync(base + ctx->DA.sig_chan, chan.data(), chan.size() * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(base + ctx->DA.sig_pool, pool.data(), pool.size() * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(base + ctx->DA.sig_cnt, cnts.data(), cnts.size() * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaStreamSynchronize(st));  // pageable staging: the vectors die with this call
+    ctx->sig_down = lists;
+    ctx->down_active = 0;
+    for (int e = 0; e < E; ++e) ctx->down_active += cnts[e] > 0 ? 1 : 0;
+    return DYNAMO_OK;
+}
+
 dynamo_status dynamo_export_codes(dynamo_ctx* ctx, int32_t expert, int32_t matrix, uint8_t* q, uint16_t* scale_f16,
                                   uint16_t* zero_f16, int32_t which, void* stream) {
     if (!ctx || !q || !scale_f16 || !zero_f16) return DYNAMO_ERR_NULL;
@@ -710,9 +881,15 @@ dynamo_status dynamo_export_codes(dynamo_ctx* ctx, int32_t expert, int32_t matri
     const dynamo_layer_desc& D = ctx->D;
     if (expert < 0 || expert >= D.n_experts + D.n_shared || matrix < 0 || matrix > 2 || which < 0 || which > 2)
         return DYNAMO_ERR_SHAPE;
-    if (which != DYNAMO_CODES_BASE && (matrix == DYNAMO_MAT_DOWN || !ctx->host_layer.ex[expert].switchable))
-        return DYNAMO_ERR_BITS;
+    if (which != DYNAMO_CODES_BASE && !ctx->host_layer.ex[expert].switchable) return DYNAMO_ERR_BITS;
     const long long n_elems = (long long)D.d_model * D.d_ff;
+    if (which != DYNAMO_CODES_BASE && matrix == DYNAMO_MAT_DOWN) {
+        if (!ctx->down_arena) return DYNAMO_ERR_STATE;  // no d_ff-side cache packed
+        CUDA_TRY(launch_export_down((const LayerDev*)ctx->arena, (const DownDev*)ctx->down_arena, expert, which, n_elems,
+                                    q, scale_f16, zero_f16, (cudaStream_t)stream));
+        ctx->launches += 1;
+        return DYNAMO_OK;
+    }
     CUDA_TRY(launch_export((const LayerDev*)ctx->arena, expert, matrix, which, n_elems, q, scale_f16, zero_f16,
                            (cudaStream_t)stream));
     ctx->launches += 1;
@@ -728,6 +905,7 @@ dynamo_status dynamo_expert_stream_bytes(dynamo_ctx* ctx, int32_t expert, size_t
     const size_t blocks = (2 * f / RB) * (d / KC) + (d / RB) * (f / KC);
     size_t b = blocks * (size_t)block_bytes(ctx->bits[expert], D.group_size);
     if (expert < D.n_experts && ctx->bits[expert] < HI_BITS) b += 2 * f * ctx->sig[expert].size() * 2;
+    if (expert < D.n_experts && ctx->down_arena) b += d * ctx->sig_down[expert].size() * 2;
     *bytes = b;
     return DYNAMO_OK;
 }

@@ -47,6 +47,23 @@ struct LayerDev {
     ExpertDev ex[MAX_EXPERTS];
 };
 
+// Significant set on the d_ff side (Section IV-B applied to the input channels of W_down, the hidden units), kept
+// in its own caller-owned arena so that layers that do not use it pay nothing.
+struct DownExpertDev {
+    uint32_t* s8m8;          // [d][f/G] half2 {scale, zero} of the 8-bit quantization of W_down
+    uint8_t* q8;             // [P2][d] 8-bit codes of the cached channels
+    __half* delta;           // [P2][d] fp16(8-bit value - base value): what a significant channel adds to the base GEMM
+    __nv_bfloat16* cache_w;  // [P2][d] bf16 originals of the cached channels (the channel cache)
+};
+struct DownDev {
+    int32_t P2, S2;
+    int32_t* cache_idx;  // [E][P2] sorted hidden-unit indices (cache headers)
+    int32_t* sig_chan;   // [E][S2] hidden unit of slot i (-1 = empty)
+    int32_t* sig_pool;   // [E][S2] pool position of slot i
+    int32_t* sig_cnt;    // [E]
+    DownExpertDev ex[MAX_EXPERTS];
+};
+
 // Workspace pointers of one forward (passed to kernels by value).
 struct WsDev {
     int32_t* counts;      // [E_tot]

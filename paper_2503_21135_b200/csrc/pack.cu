@@ -6,27 +6,9 @@
 // The double -> fp16 conversions are single roundings (cvt.rn.f16.f64).
 #include "common.cuh"
 #include "layout.cuh"
+#include "quant.cuh"
 
 namespace dyn {
-
-__device__ __forceinline__ double bf16_to_double(__nv_bfloat16 v) { return (double)__bfloat162float(v); }
-
-__device__ __forceinline__ void group_params(double lo, double hi, int bits, __half& s_h, __half& m_h, double& s,
-                                             double& m) {
-    const double L = (double)((1 << bits) - 1);
-    s_h = __double2half(__ddiv_rn(__dsub_rn(hi, lo), L));
-    if (__half2float(s_h) == 0.0f) s_h = __float2half(1.0f);
-    m_h = __double2half(lo);
-    s = (double)__half2float(s_h);
-    m = (double)__half2float(m_h);
-}
-
-__device__ __forceinline__ int quantize_code(double w, double s, double m, int bits) {
-    double t = rint(__ddiv_rn(__dsub_rn(w, m), s));
-    const double L = (double)((1 << bits) - 1);
-    t = t < 0.0 ? 0.0 : (t > L ? L : t);
-    return (int)t;
-}
 
 // One CTA packs one block (256 rows x 128 k).  Thread r owns row r of the block.
 // src_a / src_b: row-major [rows_src, K] bf16; for the fused gate/up matrix (fused = 1) rows 0..7 of

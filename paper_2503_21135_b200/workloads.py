@@ -37,6 +37,7 @@ BASE_SEED = 250321135
 
 # tensor ids of the per-stream seeds
 _T_X, _T_LOGITS, _T_OUTLIER, _T_POOL, _T_SIG, _T_BITS, _T_SWITCH, _T_ROUTER = 0, 1, 2, 3, 4, 5, 6, 7
+_T_POOL_DOWN, _T_SIG_DOWN = 8, 9
 _T_WGATE, _T_WUP, _T_WDOWN = 10, 11, 12
 
 
@@ -192,6 +193,20 @@ def cache_pool(cfg: MoEConfig, layer: int = 0) -> np.ndarray:
         extra = _rng(cfg, layer, _T_POOL, e).permutation(rest)[: cfg.cache_size - len(o)]
         out[e] = np.sort(np.concatenate([o, extra]).astype(np.int32))
     return out
+
+
+def cache_pool_down(cfg: MoEConfig, size: int, layer: int = 0) -> np.ndarray:
+    """Cached hidden units (input channels of W_down) per routed expert, int32 [E, size], each row sorted, unique."""
+    out = np.empty((cfg.n_experts, size), dtype=np.int32)
+    for e in range(cfg.n_experts):
+        out[e] = np.sort(_rng(cfg, layer, _T_POOL_DOWN, e).permutation(cfg.d_ff)[:size].astype(np.int32))
+    return out
+
+
+def sig_sets_down(cfg: MoEConfig, pool_down: np.ndarray, n_sig: int, layer: int = 0, event: int = 0) -> List[np.ndarray]:
+    """A significant set of n_sig cached hidden units per routed expert (a different draw per event)."""
+    return [np.sort(_rng(cfg, layer, _T_SIG_DOWN, e * 4096 + event).permutation(pool_down[e])[:n_sig].astype(np.int32))
+            for e in range(cfg.n_experts)]
 
 
 def initial_sig_sets(cfg: MoEConfig, pool: np.ndarray, layer: int = 0) -> List[np.ndarray]:

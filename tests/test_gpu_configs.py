@@ -54,6 +54,21 @@ def test_prefill_config():
     assert counts[7] == counts.max() and counts[7] > 2 * counts[0]        # Zipf skew: expert 7 most loaded
     # a ragged token count that leaves partial 32-token chunks in every expert
     _check_forward(cfg, gpu, ora, 1000, 48, step=1)
+    # significant hidden units on the d_ff side at full size (P2 = 128 cached, 64 significant per expert):
+    # prefill (tcgen05 pair kernel wrote h as operand tiles) and a decode-sized batch (streaming layout)
+    pool_d = wl.cache_pool_down(cfg, 128)
+    sets_d = wl.sig_sets_down(cfg, pool_d, 64)
+    gpu.pack_down_cache(wd.cuda(), bits, pool_d, 64)
+    ora.enable_down_side(oracle.as_u16(wd))
+    gpu.set_channel_switch_down(sets_d)
+    ora.set_channel_switch_down(sets_d)
+    q, s, m = gpu.export_codes(0, binding.MAT_DOWN, binding.CODES_HI_ACTIVE)
+    expect = np.zeros_like(ora.hi_down[0].q)
+    expect[:, sets_d[0]] = ora.hi_down[0].q[:, sets_d[0]]
+    assert torch.equal(q.cpu(), torch.from_numpy(expect))
+    assert np.array_equal(s.cpu().numpy().view(np.uint16), ora.hi_down[0].s)
+    _check_forward(cfg, gpu, ora, 4096, 64, step=2)
+    _check_forward(cfg, gpu, ora, 64, 64, step=3)
 
 
 def test_finegrained_config_with_shared_experts():

@@ -1,0 +1,136 @@
+"""GPU parity for significant channels on the d_ff side (Section IV-B applied to W_down's input channels): 8-bit codes
+and parameters of the cached hidden units bit-exact against the oracle, forwards on every FFN kernel within the output
+tolerance, state = last set installed, error cases."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import make_gpu_layer, make_inputs, make_oracle_layer, rel_err
+from paper_2503_21135_b200 import binding
+from paper_2503_21135_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+CFG = wl.CONFIGS["tiny"]
+P2, S2 = 96, 48
+ERR = binding.STATUS_NAMES.index
+
+
+def _u16(t):
+    return t.cpu().numpy().view(np.uint16)
+
+
+@pytest.fixture(scope="module")
+def lay():
+    wg, wu, wd, bits, pool, sets = make_inputs(CFG)
+    ora = make_oracle_layer(CFG, wg, wu, wd, bits)
+    gpu = make_gpu_layer(CFG, wg, wu, wd, bits, pool, max_tokens=256)
+    gpu.set_channel_switch(sets)
+    ora.set_channel_switch(sets)
+    pool_d = wl.cache_pool_down(CFG, P2)
+    ora.enable_down_side(oracle.as_u16(wd))
+    gpu.pack_down_cache(wd.cuda(), bits, pool_d, S2)
+    torch.cuda.synchronize()
+    return dict(bits=bits, pool_d=pool_d, ora=ora, gpu=gpu, wd=wd)
+
+
+def _forward(lay, T, step):
+    x, lg = wl.activations(CFG, T, step=step), wl.router_logits(CFG, T, step=step)
+    y = lay["gpu"].forward(x.cuda(), lg.cuda(), binding.F32)
+    torch.cuda.synchronize()
+    assert lay["gpu"].poll_status() == 0
+    ref = lay["ora"].forward(oracle.as_u16(x), lg.numpy())["y"]
+    return y, ref
+
+
+def _install(lay, sets):
+    lay["gpu"].set_channel_switch_down(sets)
+    lay["ora"].set_channel_switch_down(sets)
+
+
+def test_down_pool_codes_bit_exact(lay):
+    gpu, ora, pool_d = lay["gpu"], lay["ora"], lay["pool_d"]
+    sets = wl.sig_sets_down(CFG, pool_d, S2)
+    _install(lay, sets)
+    for e in range(CFG.n_experts):
+        if lay["bits"][e] >= 8:
+            with pytest.raises(binding.DynamoError):
+                gpu.export_codes(e, binding.MAT_DOWN, binding.CODES_HI_POOL)
+            continue
+        ref = ora.hi_down[e]
+        for which, cols in ((binding.CODES_HI_POOL, pool_d[e]), (binding.CODES_HI_ACTIVE, sets[e])):
+            q, s, m = gpu.export_codes(e, binding.MAT_DOWN, which)
+            expect = np.zeros_like(ref.q)
+            expect[:, cols] = ref.q[:, cols]
+            assert np.array_equal(q.cpu().numpy(), expect), (e, which)
+            assert np.array_equal(_u16(s), ref.s) and np.array_equal(_u16(m), ref.m), (e, which)
+    _install(lay, [np.array([], np.int32)] * CFG.n_experts)
+
+
+@pytest.mark.parametrize("T", [1, 8, 40, 200])
+def test_forward_with_down_side_sets(lay, T):
+    # T <= 64: every expert on the streaming kernel; 200: loaded experts on the tcgen05 pair kernel
+    y0, ref0 = _forward(lay, T, step=T)
+    assert rel_err(y0.cpu().numpy(), ref0) <= TOL
+    sets = wl.sig_sets_down(CFG, lay["pool_d"], S2, event=T)
+    _install(lay, sets)
+    y1, ref1 = _forward(lay, T, step=T)
+    assert rel_err(y1.cpu().numpy(), ref1) <= TOL
+    # the correction itself is resolved: GPU and oracle agree on what the sets change, far below the change
+    dg, dr = (y1 - y0).cpu().numpy().astype(np.float64), ref1 - ref0
+    assert np.max(np.abs(dr)) > 0
+    assert np.max(np.abs(dg - dr)) <= 0.05 * np.max(np.abs(dr)) + 1e-3 * np.sqrt(np.mean(ref1 ** 2))
+    # state depends only on the last set installed; the empty set is the base forward, bit for bit
+    _install(lay, wl.sig_sets_down(CFG, lay["pool_d"], 7, event=99))
+    _install(lay, sets)
+    assert torch.equal(_forward(lay, T, step=T)[0], y1)
+    _install(lay, [np.array([], np.int32)] * CFG.n_experts)
+    assert torch.equal(_forward(lay, T, step=T)[0], y0)
+
+
+def test_other_kernels_and_all_cached_units(lay):
+    gpu = lay["gpu"]
+    sets = [p[:S2] for p in lay["pool_d"]]
+    _install(lay, sets)
+    try:
+        gpu.set_prefill_kernel(binding.PREFILL_SINGLE)
+        y, ref = _forward(lay, 200, step=3)
+        assert rel_err(y.cpu().numpy(), ref) <= TOL
+        gpu.set_prefill_kernel(binding.PREFILL_PAIR)
+        gpu.set_decode_kernel(binding.DECODE_TENSOR)
+        y, ref = _forward(lay, 33, step=4)
+        assert rel_err(y.cpu().numpy(), ref) <= TOL
+    finally:
+        gpu.set_prefill_kernel(binding.PREFILL_PAIR)
+        gpu.set_decode_kernel(binding.DECODE_STREAM)
+        _install(lay, [np.array([], np.int32)] * CFG.n_experts)
+
+
+def test_down_side_errors_leave_state(lay):
+    gpu, pool_d = lay["gpu"], lay["pool_d"]
+    E = CFG.n_experts
+    sets = wl.sig_sets_down(CFG, pool_d, 5)
+    _install(lay, sets)
+    y, _ = _forward(lay, 16, step=7)
+    not_cached = np.setdiff1d(np.arange(CFG.d_ff), pool_d[0])[:1]
+    for bad, code in ((not_cached, "ERR_NOT_CACHED"), (np.array([CFG.d_ff]), "ERR_INDEX_RANGE"),
+                      (np.array([pool_d[0][0], pool_d[0][0]]), "ERR_INDEX_DUP"), (pool_d[0][: S2 + 1], "ERR_INDEX_RANGE")):
+        s = list(sets)
+        s[0] = bad
+        with pytest.raises(binding.DynamoError) as ei:
+            gpu.set_channel_switch_down(s)
+        assert ei.value.status == ERR(code), code
+    assert torch.equal(_forward(lay, 16, step=7)[0], y)
+    fresh = binding.DynamoLayer.from_config(CFG, max_tokens=16)
+    fresh.max_sig_down = S2
+    with pytest.raises(binding.DynamoError) as ei:
+        fresh.set_channel_switch_down(sets)
+    assert ei.value.status == ERR("ERR_STATE")
+    unsorted = pool_d.copy()
+    unsorted[1, [0, 1]] = unsorted[1, [1, 0]]
+    with pytest.raises(binding.DynamoError) as ei:
+        gpu.pack_down_cache(lay["wd"].cuda(), lay["bits"], unsorted, S2)
+    assert ei.value.status == ERR("ERR_INDEX_DUP")
+    assert torch.equal(_forward(lay, 16, step=7)[0], y)      # the failed re-pack left the cache in place
+    _install(lay, [np.array([], np.int32)] * E)
