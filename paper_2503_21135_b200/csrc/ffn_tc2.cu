@@ -12,9 +12,10 @@
 // Per CTA (rank r = 0 leader, 1 peer), 18 warps:
 //   warp 16 producer : bulk copies of the CTA's half block (codes of atoms 8r..8r+7, params of rows 128r..)
 //                      and of ITS half of the token tile (N/2 tokens: the B operand is split across the pair).
-//   warps 0-15 dequant: (atom, 64-k half) each: packed codes -> full fp16 weight (AND-OR, HSUB2, HFMA2 per
-//                      register pair, the weight s*q+m rounded once) -> tcgen05.st into the CTA's tensor memory;
-//                      then arrive on the LEADER's a_full barrier (remote arrive for the peer).
+//   warps 0-15 dequant: a whole atom (16 rows x 128 k) of every OTHER stage each (eight warps per stage): packed
+//                      codes -> full fp16 weight (AND-OR, HSUB2, HFMA2 per register pair, the weight s*q+m rounded
+//                      once) -> tcgen05.st into the CTA's tensor memory; then arrive on the LEADER's a_full
+//                      barrier (remote arrive for the peer).
 //   warp 17 MMA      : in the leader only: waits for both CTAs' A buffers, issues the eight MMAs of the stage
 //                      for the pair, commits (multicast) to both CTAs' a_empty / ring-slot / d_full barriers.
 //   epilogue         : warps 0-15 of each CTA read their CTA's 128 accumulator rows x N tokens (tcgen05.ld),
