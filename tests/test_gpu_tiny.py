@@ -241,3 +241,42 @@ def test_all_channels_switched_equals_uniform_8bit():
     x, lg = wl.activations(cfg, 16), wl.router_logits(cfg, 16)
     y = low.forward(x.cuda(), lg.cuda()).cpu().numpy()
     assert rel_err(y, ora.forward(oracle.as_u16(x), lg.numpy())["y"]) <= TOL
+
+
+def test_forward_can_be_captured_in_a_cuda_graph(tiny):
+    # a forward allocates nothing, synchronises nothing and zeroes its own work counters on the device, so a decode
+    # step can be captured once and replayed; inputs are read from the captured buffers at replay time
+    gpu = tiny["gpu"]
+    gpu.set_channel_switch(tiny["sets"])
+    T = 24
+    x = wl.activations(CFG, T, step=11).cuda()
+    lg = wl.router_logits(CFG, T, step=11).cuda()
+    y_ref = gpu.forward(x, lg, binding.F32).clone()
+    xs, ls = torch.zeros_like(x), torch.zeros_like(lg)
+    ys = torch.empty((T, CFG.d_model), dtype=torch.float32, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        gpu.forward(xs, ls, binding.F32, y=ys)                 # warm-up on the capture stream
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    n0 = gpu.kernel_launches()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        gpu.forward(xs, ls, binding.F32, y=ys)
+    per_forward = gpu.kernel_launches() - n0
+    assert per_forward == 6
+    xs.copy_(x)
+    ls.copy_(lg)
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(ys, y_ref)
+    x2 = wl.activations(CFG, T, step=12).cuda()
+    lg2 = wl.router_logits(CFG, T, step=12).cuda()
+    xs.copy_(x2)
+    ls.copy_(lg2)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(ys, gpu.forward(x2, lg2, binding.F32))
+    assert gpu.poll_status() == 0
