@@ -61,7 +61,8 @@ struct T2Params {
 };
 
 struct T2Bars {
-    uint64_t full[T2_NS], empty[T2_NS];  // per CTA: bytes landed / slot free again (commit from the leader)
+    uint64_t full[T2_NS], empty[T2_NS];  // per CTA: weight bytes landed / slot free again (commit from the leader)
+    uint64_t fullx[T2_NS];               // per CTA: operand bytes landed (the dequant warps need only the weights)
     uint64_t a_full[T2_NA];              // leader only: the 16 dequant warps of the pair that own the stage stored A buffer b
     uint64_t a_empty[T2_NA];                // per CTA: the MMAs that read A buffer b are done (commit)
     uint64_t d_full;                     // per CTA: the item's accumulators are complete (commit)
@@ -205,6 +206,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
     if (threadIdx.x == 0) {
         for (int i = 0; i < T2_NS; ++i) {
             mbar_init(&B->full[i], 1);
+            mbar_init(&B->fullx[i], 1);
             mbar_init(&B->empty[i], 1);
         }
         for (int i = 0; i < T2_NA; ++i) {
@@ -250,27 +252,30 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
                 if (lane == 0) {
                     if (it < n_kc) {
                         const uint8_t* blk = w.wbase + (size_t)it * w.blk_bytes;
-                        mbar_arrive_expect_tx(&B->full[s], (uint32_t)(code_half + prm_half + w.n_rg_mine * TC_RG_STRIDE));
+                        // the weights (small) first and on their own barrier: dequantization starts while the
+                        // operand tile, four times the bytes, is still on its way
+                        mbar_arrive_expect_tx(&B->full[s], (uint32_t)(code_half + prm_half));
                         bulk_g2s(st, blk + rank * code_half, (uint32_t)code_half, &B->full[s]);
                         bulk_g2s(st + code_half, blk + block_code_bytes(w.bits) + rank * prm_half, (uint32_t)prm_half,
                                  &B->full[s]);
+                        mbar_arrive_expect_tx(&B->fullx[s], (uint32_t)(w.n_rg_mine * TC_RG_STRIDE));
                         if (w.n_rg_mine > 0)
                             bulk_g2s(st + T2_WHALF_MAX, xbase + act_off(it, 8 * w.rg_mine0, p.ws.Rcap),
-                                     (uint32_t)(w.n_rg_mine * TC_RG_STRIDE), &B->full[s]);
+                                     (uint32_t)(w.n_rg_mine * TC_RG_STRIDE), &B->fullx[s]);
                     } else {
                         // cached-channel stage: up to 64 pool columns (whole 256-row tiles: this CTA uses its 128
                         // rows of them) + this CTA's token half of the operand, one copy per 32 columns
                         const int c0 = 64 * (it - n_kc), ngr = min(2, (P_pad - c0) >> 5);
-                        mbar_arrive_expect_tx(&B->full[s],
-                                              (uint32_t)(ngr * POOL_GROUP * POOL_TILE_PITCH + ngr * w.n_rg_mine * 512));
+                        mbar_arrive_expect_tx(&B->full[s], (uint32_t)(ngr * POOL_GROUP * POOL_TILE_PITCH));
                         bulk_g2s(st, reinterpret_cast<const uint8_t*>(w.ex->pool_hi) + pool_tile_off(w.rb, c0, P_pad),
                                  (uint32_t)(ngr * POOL_GROUP * POOL_TILE_PITCH), &B->full[s]);
+                        mbar_arrive_expect_tx(&B->fullx[s], (uint32_t)(ngr * w.n_rg_mine * 512));
                         if (w.n_rg_mine > 0)
                             for (int j = 0; j < ngr; ++j)
                                 bulk_g2s(st + T2_POOL_TILES + j * T2_POOL_XG,
                                          reinterpret_cast<const uint8_t*>(p.ws.xsig) +
                                              xpool_off((c0 >> 5) + j, 8 * w.rg_mine0, p.ws.Rcap),
-                                         (uint32_t)(w.n_rg_mine * 512), &B->full[s]);
+                                         (uint32_t)(w.n_rg_mine * 512), &B->fullx[s]);
                     }
                 }
                 __syncwarp();
@@ -373,6 +378,9 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
                     }
                 }
                 tc_wait_st();
+                // the arrive below also vouches for this CTA's half of the operand tile (the MMA reads both halves)
+                ok = mbar_wait_bounded(&B->fullx[s], ph, poison, status);
+                if (!ok) break;
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {  // the barrier lives in the leader: a plain arrive there, a remote one from the peer
