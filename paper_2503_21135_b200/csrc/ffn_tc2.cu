@@ -9,15 +9,19 @@
 //
 // Work item of a cluster = (expert, 256-row weight block, tile of <= 256 tokens), K over the whole input axis;
 // items are dealt round-robin over the clusters; ring, A buffers, accumulators live across items.
-// Per CTA (rank r = 0 leader, 1 peer), 18 warps:
-//   warp 16 producer : bulk copies of the CTA's half block (codes of atoms 8r..8r+7, params of rows 128r..)
-//                      and of ITS half of the token tile (N/2 tokens: the B operand is split across the pair).
+// Per CTA (rank r = 0 leader, 1 peer), 19 warps:
+//   warp 16 weights  : bulk copies of the CTA's half block (codes of atoms 8r..8r+7, params of rows 128r..) into a
+//                      ring of two small slots; a slot goes back as soon as the stage's warps hold its codes.
+//   warp 18 operands : bulk copy of ITS half of the token tile (N/2 tokens: the B operand is split across the
+//                      pair) into a ring of FIVE 36 KB slots, freed by the MMAs' commit.  The operand copy is the long
+//                      pole of a stage (2000-2800 cycles under load), so it gets the depth; the weights land on
+//                      their own barrier and are dequantized while the tile is still in flight.
 //   warps 0-15 dequant: a whole atom (16 rows x 128 k) of every OTHER stage each (eight warps per stage): packed
 //                      codes -> full fp16 weight (AND-OR, HSUB2, HFMA2 per register pair, the weight s*q+m rounded
-//                      once) -> tcgen05.st into the CTA's tensor memory; then arrive on the LEADER's a_full
-//                      barrier (remote arrive for the peer).
+//                      once) -> tcgen05.st into the CTA's tensor memory; then wait for the CTA's operand tile and
+//                      arrive on the LEADER's a_full barrier (remote arrive for the peer).
 //   warp 17 MMA      : in the leader only: waits for both CTAs' A buffers, issues the eight MMAs of the stage
-//                      for the pair, commits (multicast) to both CTAs' a_empty / ring-slot / d_full barriers.
+//                      for the pair, commits (multicast) to both CTAs' a_empty / operand-slot / d_full barriers.
 //   epilogue         : warps 0-15 of each CTA read their CTA's 128 accumulator rows x N tokens (tcgen05.ld),
 //                      SwiGLU -> fp16 h as the down GEMM's operand tiles, or fp32 rows out; then arrive on the
 //                      leader's d_empty barrier.
@@ -34,19 +38,24 @@
 namespace dyn {
 
 constexpr int T2_DEQ_WARPS = 16;
-constexpr int T2_W_PROD = 16, T2_W_MMA = 17;
-constexpr int T2_THREADS = 18 * 32;
+constexpr int T2_W_PROD = 16, T2_W_MMA = 17, T2_W_PRODX = 18;
+constexpr int T2_THREADS = 19 * 32;
 constexpr int T2_N = 256;                              // tokens per work item (128 per CTA)
 constexpr int T2_WHALF_MAX = 17408;                    // half of the largest packed block (8-bit, G = 64)
 constexpr int T2_XTILE = 16 * TC_RG_STRIDE;            // 128 tokens x 128 k: 16 row-group tiles at their buffer pitch
-constexpr int T2_STAGE_BYTES = T2_WHALF_MAX + T2_XTILE;
-constexpr int T2_POOL_TILES = 2 * POOL_GROUP * POOL_TILE_PITCH;   // cached-channel stage: 64 column tiles ...
-constexpr int T2_POOL_XG = 16 * 512;                              // ... and per 32 columns an operand tile of 16 row groups
-static_assert(T2_POOL_TILES + 2 * T2_POOL_XG <= T2_STAGE_BYTES, "cached-channel stage does not fit a ring slot");
-constexpr int T2_NS = 4;
+constexpr int T2_POOL_TILES = POOL_GROUP * POOL_TILE_PITCH;       // cached-channel stage: 32 column tiles in a weight slot ...
+constexpr int T2_POOL_XG = 16 * 512;                              // ... and their operand tile of 16 row groups in an operand slot
+static_assert(T2_POOL_TILES <= T2_WHALF_MAX && T2_POOL_XG <= T2_XTILE, "cached-channel stage does not fit its slots");
+// Two rings.  The operand tiles (36 KB, read by the MMAs, the long pole of a stage: their copy takes 2000-2800
+// cycles under load) get FIVE slots; the packed weights (read only by the dequant warps, and only at the start of
+// their visit) get two small ones that are handed back as soon as the codes are in registers.
+constexpr int T2_NW = 2;
+constexpr int T2_NX = 5;
 constexpr int T2_OFF_PREFIX = 256;                     // item prefix table: MAX_EXPERTS + 1 ints
 constexpr int T2_OFF_STAGE = 2048;
-constexpr int T2_SMEM_BYTES = T2_OFF_STAGE + T2_NS * T2_STAGE_BYTES;
+constexpr int T2_OFF_XRING = T2_OFF_STAGE + T2_NW * T2_WHALF_MAX;
+constexpr int T2_SMEM_BYTES = T2_OFF_XRING + T2_NX * T2_XTILE;
+static_assert(T2_OFF_XRING % 1024 == 0 && T2_XTILE % 1024 == 0, "operand slots must stay 1024-byte aligned");
 static_assert(T2_OFF_PREFIX + (MAX_EXPERTS + 1) * 4 <= T2_OFF_STAGE, "item table overlaps the stage ring");
 static_assert(T2_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 constexpr uint32_t T2_TMEM_COLS = 512;
@@ -61,8 +70,8 @@ struct T2Params {
 };
 
 struct T2Bars {
-    uint64_t full[T2_NS], empty[T2_NS];  // per CTA: weight bytes landed / slot free again (commit from the leader)
-    uint64_t fullx[T2_NS];               // per CTA: operand bytes landed (the dequant warps need only the weights)
+    uint64_t full[T2_NW], empty[T2_NW];    // per CTA: weight bytes landed / the stage's 8 dequant warps hold the codes
+    uint64_t fullx[T2_NX], emptyx[T2_NX];  // per CTA: operand bytes landed / the MMAs that read them are done (commit)
     uint64_t a_full[T2_NA];              // leader only: the 16 dequant warps of the pair that own the stage stored A buffer b
     uint64_t a_empty[T2_NA];                // per CTA: the MMAs that read A buffer b are done (commit)
     uint64_t d_full;                     // per CTA: the item's accumulators are complete (commit)
@@ -104,14 +113,15 @@ __device__ __forceinline__ T2Item t2_decode_item(const T2Params& p, const int* p
     it.blk_bytes = it.ex->blk_bytes;
     it.wbase = (GATEUP ? it.ex->w13 : it.ex->w2) + (size_t)it.rb * n_kc * it.blk_bytes;
     const int sig_cnt = (GATEUP && it.ex->switchable) ? L->sig_cnt[e] : 0;
-    it.n_it = n_kc + (sig_cnt > 0 ? (L->P_pad + 63) >> 6 : 0);  // + cached-channel stages of 64 pool columns
+    it.n_it = n_kc + (sig_cnt > 0 ? L->P_pad >> 5 : 0);  // + cached-channel stages of 32 pool columns
     return it;
 }
 
 // One (atom, 64-k half) of the CTA's half block -> 32 columns of the A buffer.  a_l: atom within the half
 // block (its params are rows 16*a_l .. of the half block's parameter table).
 template <int BITS>
-__device__ __forceinline__ void t2_dequant_half(const uint8_t* st, uint32_t a_cols, int a_l, int half, int lane, int G) {
+__device__ __forceinline__ void t2_dequant_half(const uint8_t* st, uint32_t a_cols, int a_l, int half, int lane, int G,
+                                                uint64_t* release) {
     const int gid = lane >> 2;
     const int ngrp = KC / G;
     constexpr int BIAS = BITS == 2 ? 4 : (BITS == 3 ? 3 : (BITS == 4 ? 2 : 0));
@@ -133,6 +143,11 @@ __device__ __forceinline__ void t2_dequant_half(const uint8_t* st, uint32_t a_co
         for (int i = 0; i < NOFF; ++i)  // zero-point times 2^(o - bias), exact
             M2[rh][i] =
                 __half2half2(__hmul(__high2half(pp), __ushort_as_half((unsigned short)((15 + OSTEP * i - BIAS) << 10))));
+    }
+    // codes and parameters are in registers: the weight slot can go back to the producer (second half only)
+    if (release) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(release);
     }
     uint32_t regs[16];
     auto step = [&](auto S4c) {
@@ -174,7 +189,8 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
 
     T2Bars* B = reinterpret_cast<T2Bars*>(smem);
     int* prefix = reinterpret_cast<int*>(smem + T2_OFF_PREFIX);
-    uint8_t* stages = smem + T2_OFF_STAGE;
+    uint8_t* wring = smem + T2_OFF_STAGE;
+    uint8_t* xring = smem + T2_OFF_XRING;
 
     // Item table (identical in both CTAs of the pair): experts above the row threshold contribute
     // (256-token tiles x row blocks) items.
@@ -204,10 +220,13 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
     if (cluster_id >= total) return;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < T2_NS; ++i) {
+        for (int i = 0; i < T2_NW; ++i) {
             mbar_init(&B->full[i], 1);
+            mbar_init(&B->empty[i], T2_DEQ_WARPS / 2);
+        }
+        for (int i = 0; i < T2_NX; ++i) {
             mbar_init(&B->fullx[i], 1);
-            mbar_init(&B->empty[i], 1);
+            mbar_init(&B->emptyx[i], 1);
         }
         for (int i = 0; i < T2_NA; ++i) {
             mbar_init(&B->a_full[i], T2_DEQ_WARPS);  // 8 warps of each CTA per stage
@@ -237,14 +256,14 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
     uint32_t gi = 0;
 
     if (warp == T2_W_PROD) {
-        // ---------------- producer (each CTA loads its own halves) ----------------
+        // ---------------- weight producer (each CTA loads its own half block) ----------------
         bool ok = true;
         for (int g = cluster_id; g < total && ok; g += n_clusters) {
             const T2Item w = t2_decode_item<GATEUP>(p, prefix, g, cursor, n_kc, rank);
             const int code_half = 8 * atom_bytes(w.bits), prm_half = 128 * (KC / G) * 4;
             for (int it = 0; it < w.n_it && ok; ++it, ++gi) {
-                const int s = gi % T2_NS, ph = (gi / T2_NS) & 1;
-                uint8_t* st = stages + (size_t)s * T2_STAGE_BYTES;
+                const int s = gi % T2_NW, ph = (gi / T2_NW) & 1;
+                uint8_t* st = wring + (size_t)s * T2_WHALF_MAX;
                 int okl = 1;
                 if (lane == 0) okl = mbar_wait_bounded(&B->empty[s], ph ^ 1, poison, status) ? 1 : 0;
                 ok = __shfl_sync(0xffffffffu, okl, 0) != 0;
@@ -252,30 +271,16 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
                 if (lane == 0) {
                     if (it < n_kc) {
                         const uint8_t* blk = w.wbase + (size_t)it * w.blk_bytes;
-                        // the weights (small) first and on their own barrier: dequantization starts while the
-                        // operand tile, four times the bytes, is still on its way
                         mbar_arrive_expect_tx(&B->full[s], (uint32_t)(code_half + prm_half));
                         bulk_g2s(st, blk + rank * code_half, (uint32_t)code_half, &B->full[s]);
                         bulk_g2s(st + code_half, blk + block_code_bytes(w.bits) + rank * prm_half, (uint32_t)prm_half,
                                  &B->full[s]);
-                        mbar_arrive_expect_tx(&B->fullx[s], (uint32_t)(w.n_rg_mine * TC_RG_STRIDE));
-                        if (w.n_rg_mine > 0)
-                            bulk_g2s(st + T2_WHALF_MAX, xbase + act_off(it, 8 * w.rg_mine0, p.ws.Rcap),
-                                     (uint32_t)(w.n_rg_mine * TC_RG_STRIDE), &B->fullx[s]);
                     } else {
-                        // cached-channel stage: up to 64 pool columns (whole 256-row tiles: this CTA uses its 128
-                        // rows of them) + this CTA's token half of the operand, one copy per 32 columns
-                        const int c0 = 64 * (it - n_kc), ngr = min(2, (P_pad - c0) >> 5);
-                        mbar_arrive_expect_tx(&B->full[s], (uint32_t)(ngr * POOL_GROUP * POOL_TILE_PITCH));
+                        // cached-channel stage: 32 pool columns (whole 256-row tiles: this CTA uses its 128 rows)
+                        const int c0 = POOL_GROUP * (it - n_kc);
+                        mbar_arrive_expect_tx(&B->full[s], (uint32_t)T2_POOL_TILES);
                         bulk_g2s(st, reinterpret_cast<const uint8_t*>(w.ex->pool_hi) + pool_tile_off(w.rb, c0, P_pad),
-                                 (uint32_t)(ngr * POOL_GROUP * POOL_TILE_PITCH), &B->full[s]);
-                        mbar_arrive_expect_tx(&B->fullx[s], (uint32_t)(ngr * w.n_rg_mine * 512));
-                        if (w.n_rg_mine > 0)
-                            for (int j = 0; j < ngr; ++j)
-                                bulk_g2s(st + T2_POOL_TILES + j * T2_POOL_XG,
-                                         reinterpret_cast<const uint8_t*>(p.ws.xsig) +
-                                             xpool_off((c0 >> 5) + j, 8 * w.rg_mine0, p.ws.Rcap),
-                                         (uint32_t)(w.n_rg_mine * 512), &B->fullx[s]);
+                                 (uint32_t)T2_POOL_TILES, &B->full[s]);
                     }
                 }
                 __syncwarp();
@@ -283,6 +288,40 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
         }
         if (!ok && lane == 0) {
             // let copies in flight land before the CTA's shared memory goes away
+            const unsigned long long t0 = globaltimer_ns();
+            while (globaltimer_ns() - t0 < 2000000ull) {
+            }
+        }
+    } else if (warp == T2_W_PRODX) {
+        // ---------------- operand producer: this CTA's half of the token tile, one slot per stage ----------------
+        bool ok = true;
+        for (int g = cluster_id; g < total && ok; g += n_clusters) {
+            const T2Item w = t2_decode_item<GATEUP>(p, prefix, g, cursor, n_kc, rank);
+            for (int it = 0; it < w.n_it && ok; ++it, ++gi) {
+                const int s = gi % T2_NX, ph = (gi / T2_NX) & 1;
+                uint8_t* st = xring + (size_t)s * T2_XTILE;
+                int okl = 1;
+                if (lane == 0) okl = mbar_wait_bounded(&B->emptyx[s], ph ^ 1, poison, status) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, okl, 0) != 0;
+                if (!ok) break;
+                if (lane == 0) {
+                    if (it < n_kc) {
+                        mbar_arrive_expect_tx(&B->fullx[s], (uint32_t)(w.n_rg_mine * TC_RG_STRIDE));
+                        if (w.n_rg_mine > 0)
+                            bulk_g2s(st, xbase + act_off(it, 8 * w.rg_mine0, p.ws.Rcap),
+                                     (uint32_t)(w.n_rg_mine * TC_RG_STRIDE), &B->fullx[s]);
+                    } else {
+                        mbar_arrive_expect_tx(&B->fullx[s], (uint32_t)(w.n_rg_mine * 512));
+                        if (w.n_rg_mine > 0)
+                            bulk_g2s(st, reinterpret_cast<const uint8_t*>(p.ws.xsig) +
+                                             xpool_off(it - n_kc, 8 * w.rg_mine0, p.ws.Rcap),
+                                     (uint32_t)(w.n_rg_mine * 512), &B->fullx[s]);
+                    }
+                }
+                __syncwarp();
+            }
+        }
+        if (!ok && lane == 0) {
             const unsigned long long t0 = globaltimer_ns();
             while (globaltimer_ns() - t0 < 2000000ull) {
             }
@@ -303,29 +342,28 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
                 // the accumulators are free once every epilogue warp of the pair has read the previous item's
                 if (ic) ok = wait1(&B->d_empty, (ic - 1) & 1);
                 for (int it = 0; it < w.n_it && ok; ++it, ++gi) {
-                    const int s = gi % T2_NS;
+                    const int s = gi % T2_NX;
                     const int b = gi % T2_NA, bph = (gi / T2_NA) & 1;
-                    // A buffer b stored by all 32 dequant warps of the pair; they waited for their stage's bytes
+                    // A buffer b stored by the 16 dequant warps of the pair that own the stage; each also waited for
+                    // its CTA's operand tile before it arrived
                     ok = wait1(&B->a_full[b], bph);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint8_t* st = stages + (size_t)s * T2_STAGE_BYTES;
+                    const uint8_t* st = xring + (size_t)s * T2_XTILE;
                     const uint32_t a0 = tbase + T2_COL_A + 64 * b;
                     if (it < n_kc) {
-                        const uint64_t desc0 = tc_desc(smem_u32(st + T2_WHALF_MAX), 128, TC_RG_STRIDE);
+                        const uint64_t desc0 = tc_desc(smem_u32(st), 128, TC_RG_STRIDE);
 #pragma unroll
                         for (int k8 = 0; k8 < 8; ++k8)
                             tc2_mma_ts_elect(tbase, a0 + 8 * k8, desc0 + (uint64_t)(16 * k8), idesc, (it | k8) ? 1u : 0u);
                     } else {
-                        const int nsub = min(4, (P_pad - 64 * (it - n_kc)) >> 4);  // 16-column MMA steps in this stage
-                        const uint32_t xt = smem_u32(st + T2_POOL_TILES);
-                        for (int j = 0; j < nsub; ++j)
-                            // operand tile of the 32-column group j/2: [row group][k-octet 4][8][8]; step (j & 1) = two octets
-                            tc2_mma_ts_elect(tbase, a0 + 8 * j, tc_desc(xt + (j >> 1) * T2_POOL_XG + (j & 1) * 256, 128, 512),
-                                             idesc, 1u);
+                        // operand tile of the stage's 32 columns: [row group][k-octet 4][8][8]; step j = two octets
+                        const uint32_t xt = smem_u32(st);
+                        for (int j = 0; j < 2; ++j)
+                            tc2_mma_ts_elect(tbase, a0 + 8 * j, tc_desc(xt + j * 256, 128, 512), idesc, 1u);
                     }
                     tc2_commit_both_elect(&B->a_empty[b]);
-                    tc2_commit_both_elect(&B->empty[s]);
+                    tc2_commit_both_elect(&B->emptyx[s]);
                 }
                 if (ok) tc2_commit_both_elect(&B->d_full);
             }
@@ -348,9 +386,10 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
             const int bits = w.bits;
             for (int it = 0; it < w.n_it && ok; ++it, ++gi) {
                 if ((int)(gi & 1) != kh) continue;
-                const int s = gi % T2_NS, ph = (gi / T2_NS) & 1;
+                const int s = gi % T2_NW, ph = (gi / T2_NW) & 1;     // weight slot (= kh: a warp always uses the same one)
+                const int xs = gi % T2_NX, xph = (gi / T2_NX) & 1;   // operand slot
                 const int b = gi % T2_NA, bph = (gi / T2_NA) & 1;
-                const uint8_t* st = stages + (size_t)s * T2_STAGE_BYTES;
+                const uint8_t* st = wring + (size_t)s * T2_WHALF_MAX;
                 ok = mbar_wait_bounded(&B->full[s], ph, poison, status) &&
                      mbar_wait_bounded(&B->a_empty[b], bph ^ 1, poison, status);
                 if (!ok) break;
@@ -358,16 +397,15 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
                 const uint32_t a_cols = my_lanes + T2_COL_A + 64 * b;
                 if (it < n_kc) {
                     switch (bits) {
-                        case 2: t2_dequant_half<2>(st, a_cols, a_l, 0, lane, G); t2_dequant_half<2>(st, a_cols, a_l, 1, lane, G); break;
-                        case 3: t2_dequant_half<3>(st, a_cols, a_l, 0, lane, G); t2_dequant_half<3>(st, a_cols, a_l, 1, lane, G); break;
-                        case 4: t2_dequant_half<4>(st, a_cols, a_l, 0, lane, G); t2_dequant_half<4>(st, a_cols, a_l, 1, lane, G); break;
-                        default: t2_dequant_half<8>(st, a_cols, a_l, 0, lane, G); t2_dequant_half<8>(st, a_cols, a_l, 1, lane, G); break;
+                        case 2: t2_dequant_half<2>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<2>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
+                        case 3: t2_dequant_half<3>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<3>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
+                        case 4: t2_dequant_half<4>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<4>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
+                        default: t2_dequant_half<8>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<8>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
                     }
                 } else {
                     // cached-channel stage: fp16 tiles [pool column][256 rows] -> A fragments -> tensor memory;
                     const int mi = lane >> 3, r = lane & 7;
-                    const int nsub = min(4, (P_pad - 64 * (it - n_kc)) >> 4);
-                    for (int j = 0; j < nsub; ++j) {
+                    for (int j = 0; j < 2; ++j) {
                         uint32_t af[4];
                         const uint32_t addr = smem_u32(st + (j * 16 + (mi >> 1) * 8 + r) * POOL_TILE_PITCH +
                                                        (16 * atom_g + (mi & 1) * 8) * 2);
@@ -376,10 +414,12 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
                                      : "r"(addr));
                         tc_st_x1(a_cols + 8 * j, af[0], af[2], af[1], af[3]);
                     }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&B->empty[s]);  // the tiles are in registers / tensor memory
                 }
                 tc_wait_st();
                 // the arrive below also vouches for this CTA's half of the operand tile (the MMA reads both halves)
-                ok = mbar_wait_bounded(&B->fullx[s], ph, poison, status);
+                ok = mbar_wait_bounded(&B->fullx[xs], xph, poison, status);
                 if (!ok) break;
                 tc_fence_before();
                 __syncwarp();
