@@ -221,7 +221,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     }
 }
 
-// The same wait with acquire at cluster scope: for barriers that threads of the peer CTA arrive on.
+// The same wait for barriers that threads of the peer CTA arrive on (default acquire: see mbar_arrive_remote).
 __device__ __forceinline__ bool mbar_wait_bounded_cluster(uint64_t* bar, uint32_t parity, volatile int* poison,
                                                           int32_t* status) {
     if (mbar_try_wait_cluster(bar, parity)) return true;

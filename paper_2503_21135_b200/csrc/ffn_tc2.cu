@@ -11,9 +11,9 @@
 // items are dealt round-robin over the clusters; ring, A buffers, accumulators live across items.
 // Per CTA (rank r = 0 leader, 1 peer), 19 warps:
 //   warp 16 weights  : bulk copies of the CTA's half block (codes of atoms 8r..8r+7, params of rows 128r..) into a
-//                      ring of two small slots; a slot goes back as soon as the stage's warps hold its codes.
+//                      ring of four small slots; a slot goes back as soon as the stage's warps hold its codes.
 //   warp 18 operands : bulk copy of ITS half of the token tile (N/2 tokens: the B operand is split across the
-//                      pair) into a ring of FIVE 36 KB slots, freed by the MMAs' commit.  The operand copy is the long
+//                      pair) into a ring of four 36 KB slots, freed by the MMAs' commit.  The operand copy is the long
 //                      pole of a stage (2000-2800 cycles under load), so it gets the depth; the weights land on
 //                      their own barrier and are dequantized while the tile is still in flight.
 //   warps 0-15 dequant: a whole atom (16 rows x 128 k) of every OTHER stage each (eight warps per stage): packed
@@ -46,11 +46,13 @@ constexpr int T2_XTILE = 16 * TC_RG_STRIDE;            // 128 tokens x 128 k: 16
 constexpr int T2_POOL_TILES = POOL_GROUP * POOL_TILE_PITCH;       // cached-channel stage: 32 column tiles in a weight slot ...
 constexpr int T2_POOL_XG = 16 * 512;                              // ... and their operand tile of 16 row groups in an operand slot
 static_assert(T2_POOL_TILES <= T2_WHALF_MAX && T2_POOL_XG <= T2_XTILE, "cached-channel stage does not fit its slots");
-// Two rings.  The operand tiles (36 KB, read by the MMAs, the long pole of a stage: their copy takes 2000-2800
-// cycles under load) get FIVE slots; the packed weights (read only by the dequant warps, and only at the start of
-// their visit) get two small ones that are handed back as soon as the codes are in registers.
-constexpr int T2_NW = 2;
-constexpr int T2_NX = 5;
+// Two rings of four slots.  The operand tiles (36 KB, read by the MMAs; their copy is the long pole of a stage at
+// 2000-2800 cycles under load) are freed by the MMAs' commit; the packed weights (read only by the dequant warps, at
+// the start of their visit) have small slots that are handed back as soon as the codes are in registers, so the
+// weights of a warp's next visit are already there when it comes back.  (Five operand + two weight slots measured
+// 2 % slower: the weight wait of ~700 cycles per visit came back.)
+constexpr int T2_NW = 4;
+constexpr int T2_NX = 4;
 constexpr int T2_OFF_PREFIX = 256;                     // item prefix table: MAX_EXPERTS + 1 ints
 constexpr int T2_OFF_STAGE = 2048;
 constexpr int T2_OFF_XRING = T2_OFF_STAGE + T2_NW * T2_WHALF_MAX;
