@@ -69,6 +69,13 @@ def test_prefill_config():
     assert np.array_equal(s.cpu().numpy().view(np.uint16), ora.hi_down[0].s)
     _check_forward(cfg, gpu, ora, 4096, 64, step=2)
     _check_forward(cfg, gpu, ora, 64, 64, step=3)
+    # the arithmetic order is fixed (static tiles, MMAs in k order, K splits summed in order), so repeated forwards
+    # must agree bit for bit: a race between the roles of the tensor-core kernel would show up here
+    x, lg = wl.activations(cfg, 4096, 0, 7).cuda(), wl.router_logits(cfg, 4096, 0, 7).cuda()
+    y0 = gpu.forward(x, lg, binding.F32).clone()
+    for _ in range(25):
+        assert torch.equal(gpu.forward(x, lg, binding.F32), y0)
+    assert gpu.poll_status() == 0
 
 
 def test_finegrained_config_with_shared_experts():
