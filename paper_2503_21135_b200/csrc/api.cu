@@ -266,7 +266,7 @@ WsDev make_ws(const dynamo_ctx* c, int T) {
     w.Rpad = w.R + 8 * (D.n_experts + D.n_shared);
     w.Rcap = D.max_tokens * (D.top_k + D.n_shared) + 8 * (D.n_experts + D.n_shared) + ROW_PAD;
     // No expert can exceed T rows.  Up to twice the threshold the streaming kernel takes a large expert as
-    // two 32-token chunks (the second pass over its blocks hits L2), which costs less than two more launches.
+    // chunks of 24 tokens (the later passes over its blocks hit L2), which costs less than two more launches.
     w.tc_min = (c->tc_min_rows != 0x7fffffff && T > 2 * c->tc_min_rows) ? c->tc_min_rows : 0x7fffffff;
     return w;
 }
@@ -373,7 +373,7 @@ dynamo_status dynamo_set_profile_events(dynamo_ctx* ctx, void* before_gateup, vo
 dynamo_status dynamo_set_tc_min_rows(dynamo_ctx* ctx, int32_t rows) {
     if (!ctx) return DYNAMO_ERR_NULL;
     if (rows < 0) return DYNAMO_ERR_SHAPE;
-    // the streaming path handles one 32-token chunk per expert when both paths are active
+    // the streaming path handles at most 32 rows (two chunks) per expert when both paths are active
     ctx->tc_min_rows = rows == 0 ? 0x7fffffff : (rows < TC_MIN_ROWS ? rows : TC_MIN_ROWS);
     return DYNAMO_OK;
 }

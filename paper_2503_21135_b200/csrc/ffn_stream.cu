@@ -1,7 +1,7 @@
 // Streaming grouped dequant-GEMM for small token counts per expert (decode path, and the generic
 // fallback for any size): HBM-bound, judged on packed-weight bytes per second.
 //
-// PERSISTENT grid (two CTAs per SM).  A work item = one (expert, 256-row weight block, chunk of <= 32
+// PERSISTENT grid (two CTAs per SM).  A work item = one (expert, 256-row weight block, chunk of <= 24
 // tokens, K split); items are ordered heaviest bit-width first and dealt round-robin to the CTAs, so
 // every CTA walks the same kind of mix.  Inside a CTA a producer warp streams the packed blocks (codes
 // + params, contiguous per 256 x 128 block) and the matching activation slices into a shared-memory ring
@@ -14,7 +14,7 @@
 //     sum_k (s*q_k + m) x_k = (s * 2^(24-bias)) * acc + m * sum_k x_k .
 // The per-group sums of x come precomputed with the activation slice.  Codes and activations are
 // exact in fp16, so the only roundings are the fp32 accumulation and the fp16 rounding of h.
-// The number of 8-token tiles (1..4) is chosen per item from the expert's actual token count.
+// The number of 8-token tiles (1..3) is chosen per item from the expert's actual token count.
 //
 // Gate/up items: after the K loop the significant-channel correction runs as extra ring stages
 // (16 channels each): the fp16 tiles of the active cached channels are fetched through the slot ->
@@ -34,7 +34,10 @@ constexpr int CONSUMER_WARPS = 16 / APW;
 constexpr int FFN_THREADS = (CONSUMER_WARPS + 1) * 32;
 constexpr int SMEM_HEADER = 2048;     // barriers, poison flag, per-expert item prefix table
 constexpr int MAX_STAGES = 16;        // ring queue depth; the ring itself is byte-granular
-constexpr int CHUNK_TOKENS = 32;
+// Tokens per work item.  24, not 32: with at most three 8-token tiles the two accumulator sets of a warp fit the 96
+// registers that two resident CTAs leave a thread (four tiles spilled ~1.3 KB of loads per thread into the
+// loops); an expert of 25-32 rows takes a second, short pass over its blocks, which hits L2.
+constexpr int CHUNK_TOKENS = 24;
 
 struct FfnParams {
     const LayerDev* L;
@@ -292,10 +295,7 @@ __device__ __forceinline__ bool consume_dispatch(const FfnParams& p, FfnSmem* S,
     if constexpr (MAXNT8 >= 2) {
         if (MAXNT8 == 2 || nt8 == 2) return consume_item<BITS, 2, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
     }
-    if constexpr (MAXNT8 >= 4) {
-        if (nt8 == 3) return consume_item<BITS, 3, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
-        return consume_item<BITS, 4, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
-    }
+    if constexpr (MAXNT8 >= 3) return consume_item<BITS, 3, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
     return false;
 }
 
@@ -512,7 +512,7 @@ cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, in
     p.work_ctr = ws.status + (gateup ? 4 : 5);
     if (small && max_rows <= 8) return gateup ? launch_one<true, 1>(p, n_ctas, st) : launch_one<false, 1>(p, n_ctas, st);
     if (small) return gateup ? launch_one<true, 2>(p, n_ctas, st) : launch_one<false, 2>(p, n_ctas, st);
-    return gateup ? launch_one<true, 4>(p, n_ctas, st) : launch_one<false, 4>(p, n_ctas, st);
+    return gateup ? launch_one<true, 3>(p, n_ctas, st) : launch_one<false, 3>(p, n_ctas, st);
 }
 
 }  // namespace dyn
