@@ -109,6 +109,22 @@ def test_finegrained_config_with_shared_experts():
     assert np.array_equal(dbg["idx"].cpu().numpy(), idx_r)
     assert np.max(np.abs(dbg["w"].cpu().numpy().astype(np.float64) - w_rt)) <= 1e-6
     assert torch.equal(gpu.forward(x.cuda(), torch.from_numpy(lg).cuda(), binding.F32), y)
+    # significant hidden units on the d_ff side with G = 64 groups, 64 routed + 2 shared experts (the shared ones
+    # and the 8-bit ones keep no set): codes of one 2-bit and one 4-bit expert, then a ragged forward
+    pool_d = wl.cache_pool_down(cfg, 64)
+    sets_d = wl.sig_sets_down(cfg, pool_d, 32)
+    gpu.pack_down_cache(wd.cuda(), bits, pool_d, 32)
+    ora.enable_down_side(oracle.as_u16(wd))
+    gpu.set_channel_switch_down(sets_d)
+    ora.set_channel_switch_down(sets_d)
+    for e in (int(np.flatnonzero(bits[:64] == 2)[0]), int(np.flatnonzero(bits[:64] == 4)[0])):
+        q, s_, m_ = gpu.export_codes(e, binding.MAT_DOWN, binding.CODES_HI_ACTIVE)
+        expect = np.zeros_like(ora.hi_down[e].q)
+        expect[:, sets_d[e]] = ora.hi_down[e].q[:, sets_d[e]]
+        assert torch.equal(q.cpu(), torch.from_numpy(expect))
+        assert np.array_equal(s_.cpu().numpy().view(np.uint16), ora.hi_down[e].s)
+        assert np.array_equal(m_.cpu().numpy().view(np.uint16), ora.hi_down[e].m)
+    _check_forward(cfg, gpu, ora, 300, 60, step=6)
 
 
 def test_switch_stress_stack():
