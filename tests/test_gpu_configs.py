@@ -40,7 +40,7 @@ def test_prefill_config():
     cfg = wl.CONFIGS["prefill"]
     wg, wu, wd, bits, pool, sets = make_inputs(cfg)
     assert bits.tolist() == [3, 3, 3, 3, 4, 4, 4, 8]
-    gpu = make_gpu_layer(cfg, wg, wu, wd, bits, pool, max_tokens=4096)
+    gpu = make_gpu_layer(cfg, wg, wu, wd, bits, pool, max_tokens=8192)
     ora = make_oracle_layer(cfg, wg, wu, wd, bits)
     gpu.set_channel_switch(sets)
     ora.set_channel_switch(sets)
@@ -54,6 +54,8 @@ def test_prefill_config():
     assert counts[7] == counts.max() and counts[7] > 2 * counts[0]        # Zipf skew: expert 7 most loaded
     # a ragged token count that leaves partial 32-token chunks in every expert
     _check_forward(cfg, gpu, ora, 1000, 48, step=1)
+    # twice the bench size: 16384 expert rows, activation buffers of half a gigabyte (offsets beyond 2^29)
+    _check_forward(cfg, gpu, ora, 8192, 40, step=5)
     # significant hidden units on the d_ff side at full size (P2 = 128 cached, 64 significant per expert):
     # prefill (tcgen05 pair kernel wrote h as operand tiles) and a decode-sized batch (streaming layout)
     pool_d = wl.cache_pool_down(cfg, 128)
