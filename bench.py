@@ -151,7 +151,7 @@ def time_steps(fn, steps, dist_barrier):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one gate/up launch, from the ncu captures summarised
 # under profiles/ (decode shape, layer 0); None where no capture of that launch exists.
-NCU_TRAFFIC_BYTES = {("decode", 8): 466.4e6 + 4.4e6, ("decode", 64): 498.1e6 + 13.3e6}
+NCU_TRAFFIC_BYTES = {("decode", 8): 493.7e6 + 3.9e6, ("decode", 64): 501.3e6 + 15.7e6}
 
 
 def kernel_times(layers, step_fn, steps):
