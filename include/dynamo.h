@@ -40,7 +40,7 @@ typedef enum {
     DYNAMO_ERR_NULL = 1,            /* a required pointer is NULL */
     DYNAMO_ERR_SHAPE = 2,           /* a dimension violates the shape rules above */
     DYNAMO_ERR_BITS = 3,            /* a bit-width is not one of 2, 3, 4, 8 (shared experts: 8) */
-    DYNAMO_ERR_ALIGN = 4,           /* a device buffer is not 256-byte aligned */
+    DYNAMO_ERR_ALIGN = 4,           /* an arena is not 256-byte aligned, or x / y / w_router not 16-byte aligned */
     DYNAMO_ERR_ARENA_TOO_SMALL = 5, /* weights arena or workspace smaller than dynamo_arena_bytes says */
     DYNAMO_ERR_INDEX_RANGE = 6,     /* a channel index is outside [0, d_model) or a count outside [0, S] */
     DYNAMO_ERR_INDEX_DUP = 7,       /* a channel index appears twice / cache_idx not strictly increasing */
@@ -140,7 +140,7 @@ dynamo_status dynamo_set_switch_mode(dynamo_ctx* ctx, int32_t mode);
 /* Forward of the layer: router top-k -> token permutation -> mixed-precision grouped SwiGLU FFN
  * with the significant-channel correction -> weighted un-permute.  [Section II-A: Top-K expert
  * selection, one-to-many dispatch; Section V-B: packed load, dequantize, tensor-core MMA, fused.]
- *   x             : dev bf16 [T, d]
+ *   x             : dev bf16 [T, d], 16-byte aligned (as y must be; misaligned -> ERR_ALIGN)
  *   router_logits : dev fp32 [T, E]   (the router GEMM is outside this path)
  *   y             : dev [T, d], bf16 or fp32 per y_dtype
  * topk = the k largest logits (ties -> lower index), weights = softmax over all E restricted to

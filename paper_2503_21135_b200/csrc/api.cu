@@ -668,7 +668,8 @@ static dynamo_status forward_impl(dynamo_ctx* ctx, const void* x, const float* r
     if (y_dtype != DYNAMO_BF16 && y_dtype != DYNAMO_F32) return DYNAMO_ERR_SHAPE;
     if (T == 0) return DYNAMO_OK;
     if (!x || (!router_logits && !w_router) || !y) return DYNAMO_ERR_NULL;
-    if (w_router && (((uintptr_t)w_router | (uintptr_t)x) & 15)) return DYNAMO_ERR_ALIGN;  // 16-byte vector loads
+    // 16-byte vector loads of x (and of the router weights), 16-byte vector stores of y
+    if ((((uintptr_t)x | (uintptr_t)y) & 15) || (w_router && ((uintptr_t)w_router & 15))) return DYNAMO_ERR_ALIGN;
     cudaStream_t st = (cudaStream_t)stream;
     const LayerDev* L = (const LayerDev*)ctx->arena;
     WsDev ws = make_ws(ctx, T);

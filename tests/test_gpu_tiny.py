@@ -280,3 +280,18 @@ def test_forward_can_be_captured_in_a_cuda_graph(tiny):
     torch.cuda.synchronize()
     assert torch.equal(ys, gpu.forward(x2, lg2, binding.F32))
     assert gpu.poll_status() == 0
+
+
+def test_misaligned_input_or_output_is_rejected(tiny):
+    # x and y are read and written with 16-byte vectors: an address off by one element is an argument error
+    gpu = tiny["gpu"]
+    x = wl.activations(CFG, 5, step=13).cuda()
+    lg = wl.router_logits(CFG, 5, step=13).cuda()
+    y = torch.empty((5, CFG.d_model), dtype=torch.float32, device="cuda")
+    ok = binding.dynamo_moe_forward(gpu.ctx, x.data_ptr(), lg.data_ptr(), 4, y.data_ptr(), binding.F32, None, None)
+    assert ok == 0
+    for xp, yp in ((x.data_ptr() + 2, y.data_ptr()), (x.data_ptr(), y.data_ptr() + 4)):
+        st = binding.dynamo_moe_forward(gpu.ctx, xp, lg.data_ptr(), 4, yp, binding.F32, None, None)
+        assert st == binding.STATUS_NAMES.index("ERR_ALIGN")
+    torch.cuda.synchronize()
+    assert gpu.poll_status() == 0
