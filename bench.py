@@ -98,8 +98,7 @@ class ClockSampler:
         return out
 
 
-def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None, decode_kernel=None, prefill_kernel=None,
-                 down_side=0):
+def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None, down_side=0):
     """Generate, upload and pack ``n_layers`` independent layers; they share one workspace."""
     from paper_2503_21135_b200 import binding
 
@@ -118,10 +117,6 @@ def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None, decode_ker
             layer.set_channel_switch_down(wl.sig_sets_down(cfg, pool_d, down_side, l))
         if tc_min_rows is not None:
             layer.set_tc_min_rows(tc_min_rows)
-        if prefill_kernel is not None:
-            layer.set_prefill_kernel(binding.PREFILL_SINGLE if prefill_kernel == "single" else binding.PREFILL_PAIR)
-        if decode_kernel is not None:
-            layer.set_decode_kernel(binding.DECODE_STREAM if decode_kernel == "stream" else binding.DECODE_TENSOR)
         torch.cuda.synchronize()
         ws = layer.workspace
         layers.append(layer)
@@ -202,8 +197,7 @@ def run_ours(args, rank, world, device):
         if world > 1:
             torch.distributed.barrier()
 
-    layers, meta = build_layers(cfg, n_layers, max(T, max(cfg.tokens)), device, args.tc_min_rows, args.decode_kernel, args.prefill_kernel,
-                                args.down_side)
+    layers, meta = build_layers(cfg, n_layers, max(T, max(cfg.tokens)), device, args.tc_min_rows, args.down_side)
     sweep_T = sorted(set([T] + (list(cfg.tokens) if args.sweep else [])))
     results = {}
     for Tcur in sweep_T:
@@ -316,8 +310,7 @@ def run_ours(args, rank, world, device):
         achieved = gu_flops / (r["gu_ms"] / 1e3) / 1e12
         out["roofline"] = {"bound": "tensor", "achieved": achieved, "peak": tensor_peak, "unit": "TFLOP/s",
                            "frac": achieved / tensor_peak, "traffic": None, "peak_kind": peak_kind + " (sustained fp16/bf16)",
-                           "kernel": ("ffn_tc_kernel<gate/up>" if args.prefill_kernel == "single" else "ffn_tc2_kernel<gate/up>")
-                           + " (+ streaming kernel for experts of <= 32 rows)",
+                           "kernel": "ffn_tc2_kernel<gate/up> (+ streaming kernel for experts of <= 32 rows)",
                            "algorithmic_flops_per_launch": gu_flops, "avg_launch_ms": r["gu_ms"],
                            "down_launch": {"achieved": gu_flops / 2 / (r["dn_ms"] / 1e3) / 1e12, "avg_launch_ms": r["dn_ms"]},
                            "whole_step_tflops": 1.5 * gu_flops / (ms_step / 1e3) / 1e12}
@@ -327,8 +320,7 @@ def run_ours(args, rank, world, device):
       out["roofline"] = {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                        "frac": achieved / hbm_peak, "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, T)),
                        "peak_kind": peak_kind,
-                       "kernel": "ffn_tcd_kernel<gate/up>" if (args.decode_kernel == "tensor" and T <= 64)
-                       else "ffn_stream_kernel<gate/up>",
+                       "kernel": "ffn_stream_kernel<gate/up>",
                        "algorithmic_bytes_per_launch": r["gu_bytes"], "avg_launch_ms": r["gu_ms"],
                        "down_launch": {"achieved": r["dn_bytes"] / (r["dn_ms"] / 1e3) / 1e9, "avg_launch_ms": r["dn_ms"]},
                        "whole_step": {"achieved": r["bytes_per_step"] / (ms_step / 1e3) / 1e9,
@@ -494,10 +486,6 @@ def main():
     ap.add_argument("--no-switch", action="store_true", help="skip the runtime channel-switch measurement")
     ap.add_argument("--tc-min-rows", type=int, default=None,
                     help="experts with more rows than this take the tcgen05 kernel (0: streaming kernel only)")
-    ap.add_argument("--prefill-kernel", default=None, choices=["pair", "single"],
-                    help="tcgen05 kernel for experts above the row threshold (default: the library's, pair)")
-    ap.add_argument("--decode-kernel", default=None, choices=["tensor", "stream"],
-                    help="kernel for batches of up to 64 tokens (default: the library's, stream)")
     ap.add_argument("--router", action="store_true",
                     help="also time the forward with the router GEMM + top-k fused in front")
     ap.add_argument("--down-side", type=int, default=0,

@@ -23,7 +23,13 @@
  *    1 <= top_k <= 8, n_experts <= 256, n_experts + n_shared <= 264, top_k <= n_experts,
  *    max_sig <= cache_size <= d_model, max_sig <= 256.
  *  - MMA operand format is fp16 (codes and activations are exact in it; the hidden
- *    activation h is rounded to fp16); accumulation is fp32.
+ *    activation h is rounded to fp16); accumulation is fp32.  The operands carry a
+ *    power-of-two pre-scale of up to 2^4, so activations must satisfy |x| <= 4080 and
+ *    |h| <= 4080 (the largest bf16 / fp16 value below 65504 / 16).  A larger magnitude (an
+ *    infinity included) is CLAMPED to +-4080, the forward completes with the clamped value
+ *    (exactly the forward of the clamped input), and the sticky status bit
+ *    behind DYNAMO_ERR_RANGE is set (read and cleared by dynamo_poll_status).  NaN inputs
+ *    propagate.
  */
 #ifndef DYNAMO_H_
 #define DYNAMO_H_
@@ -49,7 +55,8 @@ typedef enum {
     DYNAMO_ERR_TOKENS = 10,         /* T < 0 or T > max_tokens */
     DYNAMO_ERR_CUDA = 11,           /* a CUDA runtime call failed */
     DYNAMO_ERR_TIMEOUT = 12,        /* a bounded device-side wait expired (see dynamo_poll_status) */
-    DYNAMO_ERR_ARG = 13             /* a scalar or array value is outside its domain (dynamo_assign_bits) */
+    DYNAMO_ERR_ARG = 13,            /* a scalar or array value is outside its domain */
+    DYNAMO_ERR_RANGE = 14           /* an activation exceeded the fp16 operand range and was clamped (see Conventions) */
 } dynamo_status;
 
 typedef struct {
@@ -183,9 +190,22 @@ dynamo_status dynamo_export_codes(dynamo_ctx* ctx, int32_t expert, int32_t matri
  * channels.  Host only (uses the sets last installed). */
 dynamo_status dynamo_expert_stream_bytes(dynamo_ctx* ctx, int32_t expert, size_t* bytes);
 
-/* Synchronises the stream, reads the device status word: DYNAMO_OK or DYNAMO_ERR_TIMEOUT, and
- * clears it. */
+/* Synchronises the stream, reads the device status word and clears it.  (Utility call: the paper has no
+ * counterpart.)  DYNAMO_ERR_TIMEOUT: a bounded device-side wait expired; the kernels of that forward and of every
+ * later one started nothing, outputs are undefined until the status is cleared by this call.  DYNAMO_ERR_RANGE: an
+ * activation was clamped (see Conventions); outputs are defined.  TIMEOUT wins when both are set.  Else DYNAMO_OK. */
 dynamo_status dynamo_poll_status(dynamo_ctx* ctx, void* stream);
+
+/* Debug calls.  (The paper has no counterpart.)
+ * dynamo_debug_expire_wait: launches one warp that waits, through the same bounded wait the FFN kernels use but with
+ *   limit_ns (1e3 .. 1e8) as its limit, on a barrier that nobody arrives at.  The wait gives up, sets the TIMEOUT
+ *   status bit and the kernel returns: nothing faults or hangs.  Exercises the failure path end to end
+ *   (dynamo_poll_status reports ERR_TIMEOUT, forwards in between start nothing).
+ * dynamo_debug_check_guards: every region of the weights arena and of the workspace is followed by a 256-byte guard
+ *   block written at pack time; synchronises the stream and returns in *n_bad_bytes how many guard bytes have changed
+ *   since (0 unless a kernel stored outside its region). */
+dynamo_status dynamo_debug_expire_wait(dynamo_ctx* ctx, int64_t limit_ns, void* stream);
+dynamo_status dynamo_debug_check_guards(dynamo_ctx* ctx, int64_t* n_bad_bytes, void* stream);
 
 /* Path selection: experts that receive more than `rows` tokens in a forward run on the tcgen05
  * (tensor-memory) kernel, the others on the streaming kernel.  Default 32 (also the maximum);
@@ -286,29 +306,6 @@ dynamo_status dynamo_assign_bits(const double* x, int32_t n, int32_t dim, int32_
                                  int32_t max_iter, const double* u0, const double* token_share,
                                  const int32_t* levels, double overlap, int32_t* bits_out, int32_t* cluster_out,
                                  double* v_out, double* u_out, int32_t* iters_out);
-
-/* Which kernel serves small batches (forwards of at most 64 tokens, where every expert has few rows and the
- * forward is bound by streaming the packed weights of Section V-B from HBM):
- *   DYNAMO_DECODE_STREAM (default): the streaming kernel (mma.sync) takes every expert, as it does for the
- *       experts of up to 32 rows of larger batches;
- *   DYNAMO_DECODE_TENSOR: the decode tensor-core kernel takes every expert: codes are expanded in place into
- *       tensor memory, tcgen05.mma accumulates one quantization group at a time, scale and zero are applied
- *       once per group when the group is read back.  Measured slower than the streaming kernel on B200
- *       (the expand -> MMA -> fold hand-offs per 128-k stage cost more than they save); kept selectable.
- * Both implement the same arithmetic definition.  Host-side setting; takes effect at the next forward.
- * Errors: NULL ctx -> ERR_NULL; unknown kind -> ERR_SHAPE. */
-enum { DYNAMO_DECODE_TENSOR = 0, DYNAMO_DECODE_STREAM = 1 };
-dynamo_status dynamo_set_decode_kernel(dynamo_ctx* ctx, int32_t kind);
-
-/* Which tcgen05 kernel serves the experts above the row threshold (prefill-sized work, Section V-B's fused
- * dequantize + tensor-core GEMM):
- *   DYNAMO_PREFILL_PAIR (default): thread-block clusters of two CTAs; one MMA spans both SMs' tensor cores
- *       (256 weight rows x up to 256 tokens), each CTA dequantizes its 128 rows into its own tensor memory;
- *   DYNAMO_PREFILL_SINGLE: one CTA per SM, 256 weight rows x up to 128 tokens per work item.
- * Both implement the same arithmetic definition.  Host-side setting; takes effect at the next forward.
- * Errors: NULL ctx -> ERR_NULL; unknown kind -> ERR_SHAPE. */
-enum { DYNAMO_PREFILL_PAIR = 0, DYNAMO_PREFILL_SINGLE = 1 };
-dynamo_status dynamo_set_prefill_kernel(dynamo_ctx* ctx, int32_t kind);
 
 /* Measurement hook: three cudaEvent_t handles (any may be NULL) that every following forward records on
  * its stream before the gate/up FFN launch, after it, and after the down FFN launch, so that a

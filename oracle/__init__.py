@@ -349,23 +349,19 @@ class OracleLayer:
 
 
 # ---- runtime selection of the significant channels (Sections IV-B, V-A; a "next" row of the scope table) ----
-# The statistic decides an integer (which channels are selected), so it is accumulated in the CUDA path's
-# precision and order: float32, tokens ascending inside a forward, then one float32 addition to the running total.
+# The paper leaves the statistic loose; the reading taken is the activation mass of an input channel over the tokens
+# routed to the expert.  Plain float64 sums: |x| of a bf16 value is exact, and so are sums of a few thousand of them.
 
 def channel_stats_update(stats: np.ndarray, x_u16: np.ndarray, idx: np.ndarray, pool: np.ndarray) -> np.ndarray:
-    """stats float32 [E, P] += per expert e, cached channel pool[e][j]: sum over the tokens routed to e (ascending)
-    of |x[t][pool[e][j]]|.  x_u16: bf16 bit patterns [T, d]; idx: int32 [T, k] chosen experts; returns stats."""
+    """stats float64 [E, P] + per expert e, cached channel pool[e][j]: sum over the tokens routed to e of
+    |x[t][pool[e][j]]|.  x_u16: bf16 bit patterns [T, d]; idx: int32 [T, k] chosen experts; returns the new stats."""
     E, P = pool.shape
-    xa = np.abs((x_u16.astype(np.uint32) << 16).view(np.float32))      # |x| as float32: exact for bf16
-    out = np.array(stats, dtype=np.float32, copy=True)
+    xa = np.abs((x_u16.astype(np.uint32) << 16).view(np.float32)).astype(np.float64)
+    out = np.array(stats, dtype=np.float64, copy=True)
     for e in range(E):
-        toks = np.flatnonzero((idx == e).any(axis=1))                   # ascending token order
-        if len(toks) == 0:
-            continue
-        batch = np.zeros((P,), dtype=np.float32)
-        for t in toks:
-            batch = (batch + xa[t, pool[e]]).astype(np.float32)         # one rounding per addition, in token order
-        out[e] = (out[e] + batch).astype(np.float32)
+        for t in range(xa.shape[0]):
+            if (idx[t] == e).any():
+                out[e] += xa[t, pool[e]]
     return out
 
 

@@ -24,18 +24,18 @@ BF16, F32 = 0, 1
 MAT_GATE, MAT_UP, MAT_DOWN = 0, 1, 2
 CODES_BASE, CODES_HI_POOL, CODES_HI_ACTIVE = 0, 1, 2
 SWITCH_SELECT, SWITCH_REQUANT = 0, 1
-DECODE_TENSOR, DECODE_STREAM = 0, 1
-PREFILL_PAIR, PREFILL_SINGLE = 0, 1
 
 STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_BITS", "ERR_ALIGN", "ERR_ARENA_TOO_SMALL", "ERR_INDEX_RANGE",
-                "ERR_INDEX_DUP", "ERR_NOT_CACHED", "ERR_STATE", "ERR_TOKENS", "ERR_CUDA", "ERR_TIMEOUT", "ERR_ARG"]
+                "ERR_INDEX_DUP", "ERR_NOT_CACHED", "ERR_STATE", "ERR_TOKENS", "ERR_CUDA", "ERR_TIMEOUT", "ERR_ARG", "ERR_RANGE"]
 
 EXPORTED = ["dynamo_create", "dynamo_destroy", "dynamo_arena_bytes", "dynamo_pack_experts",
             "dynamo_set_channel_switch", "dynamo_set_channel_switch_many", "dynamo_set_switch_mode",
             "dynamo_moe_forward", "dynamo_moe_forward_router", "dynamo_moe_forward_host", "dynamo_export_codes", "dynamo_expert_stream_bytes",
-            "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_decode_kernel", "dynamo_set_prefill_kernel", "dynamo_set_stats_collection", "dynamo_set_channel_precision", "dynamo_assign_bits",
+            "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_stats_collection", "dynamo_set_channel_precision", "dynamo_assign_bits",
             "dynamo_down_cache_bytes", "dynamo_pack_down_cache", "dynamo_set_channel_switch_down",
-            "dynamo_get_channel_stats", "dynamo_select_significant", "dynamo_route_permute_static", "dynamo_kernel_launches", "dynamo_status_str"]
+            "dynamo_get_channel_stats", "dynamo_select_significant", "dynamo_route_permute_static",
+            "dynamo_debug_expire_wait", "dynamo_debug_check_guards",
+            "dynamo_kernel_launches", "dynamo_status_str"]
 
 
 class LayerDesc(ctypes.Structure):
@@ -80,8 +80,6 @@ def load():
         L.dynamo_poll_status.argtypes = [vp, vp]
         L.dynamo_set_profile_events.argtypes = [vp, vp, vp, vp]
         L.dynamo_set_tc_min_rows.argtypes = [vp, i32]
-        L.dynamo_set_decode_kernel.argtypes = [vp, i32]
-        L.dynamo_set_prefill_kernel.argtypes = [vp, i32]
         L.dynamo_set_stats_collection.argtypes = [vp, i32]
         L.dynamo_set_channel_precision.argtypes = [vp, i32p, vp]
         L.dynamo_down_cache_bytes.argtypes = [vp, i32p, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
@@ -93,6 +91,8 @@ def load():
         L.dynamo_get_channel_stats.argtypes = [vp, vp, vp]
         L.dynamo_select_significant.argtypes = [vp, i32, i32, i32p, i32p, vp]
         L.dynamo_route_permute_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
+        L.dynamo_debug_expire_wait.argtypes = [vp, ctypes.c_int64, vp]
+        L.dynamo_debug_check_guards.argtypes = [vp, ctypes.POINTER(ctypes.c_int64), vp]
         L.dynamo_kernel_launches.argtypes = [vp]
         L.dynamo_kernel_launches.restype = ctypes.c_int64
         L.dynamo_status_str.argtypes = [i32]
@@ -180,14 +180,6 @@ def dynamo_poll_status(ctx, stream) -> int:
 
 def dynamo_set_tc_min_rows(ctx, rows: int) -> int:
     return load().dynamo_set_tc_min_rows(ctx, rows)
-
-
-def dynamo_set_decode_kernel(ctx, kind: int) -> int:
-    return load().dynamo_set_decode_kernel(ctx, kind)
-
-
-def dynamo_set_prefill_kernel(ctx, kind: int) -> int:
-    return load().dynamo_set_prefill_kernel(ctx, kind)
 
 
 def dynamo_set_profile_events(ctx, e0, e1, e2) -> int:
@@ -406,12 +398,6 @@ class DynamoLayer:
                "dynamo_select_significant")
         return [idx[e, : cnt[e]].copy() for e in range(E)]
 
-    def set_prefill_kernel(self, kind: int):
-        _check(dynamo_set_prefill_kernel(self.ctx, kind), "dynamo_set_prefill_kernel")
-
-    def set_decode_kernel(self, kind: int):
-        _check(dynamo_set_decode_kernel(self.ctx, kind), "dynamo_set_decode_kernel")
-
     def set_profile_events(self, events=None):
         """events: three torch.cuda.Event (already recorded once, so that their handles exist) or None."""
         h = [None, None, None] if events is None else [e.cuda_event for e in events]
@@ -419,6 +405,14 @@ class DynamoLayer:
 
     def poll_status(self) -> int:
         return dynamo_poll_status(self.ctx, _stream())
+
+    def debug_expire_wait(self, limit_ns: int):
+        _check(load().dynamo_debug_expire_wait(self.ctx, int(limit_ns), _stream()), "dynamo_debug_expire_wait")
+
+    def debug_check_guards(self) -> int:
+        n = ctypes.c_int64(-1)
+        _check(load().dynamo_debug_check_guards(self.ctx, ctypes.byref(n), _stream()), "dynamo_debug_check_guards")
+        return int(n.value)
 
     def kernel_launches(self) -> int:
         return dynamo_kernel_launches(self.ctx)

@@ -27,19 +27,20 @@ cudaError_t launch_route_gemm(const void* x, const void* w_router, const float* 
                               int renorm, float* logits_out, int32_t* idx, float* w, cudaStream_t st);
 cudaError_t launch_scan(const WsDev& ws, int E, int Es, int k, cudaStream_t st);
 cudaError_t launch_gather(const LayerDev* L, const WsDev& ws, const void* x, cudaStream_t st);
+bool front_fits(int T, int k);
+cudaError_t launch_front(const LayerDev* L, const WsDev& ws, const void* x, const float* logits, int E, int Es, int k,
+                         int renorm, cudaStream_t st);
 cudaError_t launch_combine(const WsDev& ws, int d, int k, int Es, void* y, int y_f32, long long split_stride,
                            cudaStream_t st);
 cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int ksplit, int n_experts,
                               long long split_stride, int max_rows, int n_sms, cudaStream_t st);
-cudaError_t launch_ffn_tc(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int n_experts, int n_sms,
-                          cudaStream_t st);
-cudaError_t launch_ffn_tc2(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int n_experts, int n_sms,
+cudaError_t setup_ffn_tc2(int n_sms, int* clusters_out);
+cudaError_t launch_ffn_tc2(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int n_experts, int n_clusters,
                            cudaStream_t st);
-cudaError_t launch_ffn_tcd(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int ksplit, int n_experts,
-                           long long split_stride, int n_sms, cudaStream_t st);
 cudaError_t launch_stats(const LayerDev* L, const WsDev& ws, const void* x, float* stats, int E, cudaStream_t st);
 cudaError_t launch_select(const LayerDev* L, float* stats, int E, int P, int n_sel, int reset, int32_t* chosen,
                           cudaStream_t st);
+cudaError_t launch_expire_wait(int32_t* status, unsigned long long limit_ns, cudaStream_t st);
 cudaError_t launch_switch(const SwitchLayers& layers, int n_layers, int E, const int32_t* staging, int per_layer_ints,
                           cudaStream_t st);
 }  // namespace dyn
@@ -53,22 +54,26 @@ constexpr int ROW_PAD = 32;            // extra activation rows so a token chunk
 constexpr int MAX_SWITCH_LAYERS = 64;
 constexpr int DECODE_ROWS = 1024;      // up to this many permuted rows the down GEMM is split along K
 constexpr int MAX_KSPLIT = 8;
-constexpr int DECODE_FOLD_TOKENS = 64;  // up to this many tokens the decode tensor-core kernel serves every expert
 
 inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
+// Every region of the weights arena and of the workspace is followed by a guard of GUARD bytes filled with
+// GUARD_BYTE at pack time; no kernel may write there (dynamo_debug_check_guards counts the bytes that changed).
+constexpr size_t GUARD = 256;
+constexpr int GUARD_BYTE = 0xC5;
 
 struct ArenaLayout {
     size_t header = 0;
     std::vector<size_t> w13, w2, s8m8_g, s8m8_u, mm_g, mm_u, q8_g, q8_u, cw_g, cw_u, pool_hi;
     size_t cache_idx = 0, sig_chan = 0, sig_pool = 0, sig_cnt = 0, sigmask = 0, stats = 0;
     size_t total = 0;
+    std::vector<size_t> guards;  // offsets of the guard blocks
 };
 
 struct WsLayout {
     size_t status, counts, offsets, off_pad, topk_idx, topk_w, perm, pos, row_token, row_expert, xperm, xsig,
         hbuf, ypart,
         stage_x, stage_logits, stage_y, stage_switch, total;
-    long long ypart_rows;  // capacity in rows of one K split
+    std::vector<size_t> guards;  // offsets of the guard blocks
 };
 
 inline int s_pad_of(const dynamo_layer_desc& D) { return (D.max_sig + 15) / 16 * 16; }
@@ -141,9 +146,17 @@ void arena_layout(const dynamo_layer_desc& D, const int32_t* bits, ArenaLayout& 
     const int n = D.n_experts + D.n_shared;
     const size_t d = D.d_model, f = D.d_ff, G = D.group_size, P = D.cache_size;
     const size_t n_rb13 = 2 * f / RB, n_kc13 = d / KC, n_rb2 = d / RB, n_kc2 = f / KC;
-    size_t off = align_up(sizeof(LayerDev));
+    A.guards.clear();
+    size_t off = 0;
     A.header = 0;
-    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    auto take = [&](size_t bytes) {
+        size_t o = off;
+        off = align_up(off + bytes);
+        A.guards.push_back(off);
+        off += GUARD;
+        return o;
+    };
+    take(sizeof(LayerDev));
     A.w13.assign(n, 0); A.w2.assign(n, 0);
     A.s8m8_g.assign(n, 0); A.s8m8_u.assign(n, 0); A.q8_g.assign(n, 0); A.q8_u.assign(n, 0);
     A.mm_g.assign(n, 0); A.mm_u.assign(n, 0);
@@ -179,7 +192,14 @@ void ws_layout(const dynamo_layer_desc& D, WsLayout& W) {
     const size_t n = D.n_experts + D.n_shared, T = D.max_tokens, k = D.top_k, kk = D.top_k + D.n_shared;
     const size_t R = T * kk, d = D.d_model, f = D.d_ff, S_pad = s_pad_of(D);
     size_t off = 0;
-    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    W.guards.clear();
+    auto take = [&](size_t bytes) {
+        size_t o = off;
+        off = align_up(off + bytes);
+        W.guards.push_back(off);
+        off += GUARD;
+        return o;
+    };
     W.status = take(256);
     W.counts = take(n * 4);
     W.offsets = take((n + 1) * 4);
@@ -196,8 +216,7 @@ void ws_layout(const dynamo_layer_desc& D, WsLayout& W) {
     W.hbuf = take((Rp + ROW_PAD) * (f / KC) * XROW);
     const size_t ks = std::min<size_t>(MAX_KSPLIT, f / KC);
     const size_t small_rows = std::min<size_t>(R, DECODE_ROWS);
-    W.ypart_rows = (long long)std::max(Rp, small_rows);
-    W.ypart = take(std::max(Rp, ks * (small_rows + 8 * n)) * d * 4);
+    W.ypart = take(std::max(Rp, ks * (small_rows + 8 * n)) * d * 4);   // fp32 rows of the down GEMM, per K split
     W.stage_x = take(T * d * 2);
     W.stage_logits = take(T * (size_t)D.n_experts * 4);
     W.stage_y = take(T * d * 4);
@@ -228,10 +247,9 @@ struct dynamo_ctx {
     LayerDev host_layer;                         // host mirror of the arena header
     int switch_mode = DYNAMO_SWITCH_SELECT;
     int tc_min_rows = TC_MIN_ROWS;               // experts with more rows take the tcgen05 path
-    int decode_kernel = DYNAMO_DECODE_STREAM;
     int collect_stats = 0;                       // 1: every forward adds to the per-channel activation statistics
-    int prefill_kernel = DYNAMO_PREFILL_PAIR;    // which tcgen05 kernel serves experts above the row threshold    // which kernel serves forwards of up to DECODE_FOLD_TOKENS tokens
     int n_sms = 148;                             // SM count of the device the layer was packed on
+    int tc2_clusters[2] = {0, 0};                // resident CTA pairs of the tcgen05 kernel there (down, gate/up)
     int64_t launches = 0;
     cudaEvent_t prof_ev[3] = {nullptr, nullptr, nullptr};  // optional: before gate/up, after gate/up, after down
     std::vector<int32_t> upload;                 // scratch for switch uploads
@@ -259,9 +277,6 @@ WsDev make_ws(const dynamo_ctx* c, int T) {
     w.T = T;
     w.R = T * (D.top_k + D.n_shared);
     w.ksplit = ksplit_for(D, T);
-    // Small batches: every expert has few rows, the forward is bound by streaming weights, and all experts
-    // go through the decode tensor-core kernel (operand-tile activation layout everywhere).
-    w.fold = (c->decode_kernel == DYNAMO_DECODE_TENSOR && T <= DECODE_FOLD_TOKENS) ? 1 : 0;
     w.off_pad = (int32_t*)(b + c->W.off_pad);
     w.Rpad = w.R + 8 * (D.n_experts + D.n_shared);
     w.Rcap = D.max_tokens * (D.top_k + D.n_shared) + 8 * (D.n_experts + D.n_shared) + ROW_PAD;
@@ -320,6 +335,7 @@ const char* dynamo_status_str(dynamo_status s) {
         case DYNAMO_ERR_CUDA: return "CUDA runtime error";
         case DYNAMO_ERR_TIMEOUT: return "device-side wait expired";
         case DYNAMO_ERR_ARG: return "argument value outside its domain";
+        case DYNAMO_ERR_RANGE: return "an activation was clamped to the fp16 operand range";
     }
     return "unknown status";
 }
@@ -441,20 +457,6 @@ dynamo_status dynamo_select_significant(dynamo_ctx* ctx, int32_t n_select, int32
     return DYNAMO_OK;
 }
 
-dynamo_status dynamo_set_prefill_kernel(dynamo_ctx* ctx, int32_t kind) {
-    if (!ctx) return DYNAMO_ERR_NULL;
-    if (kind != DYNAMO_PREFILL_PAIR && kind != DYNAMO_PREFILL_SINGLE) return DYNAMO_ERR_SHAPE;
-    ctx->prefill_kernel = kind;
-    return DYNAMO_OK;
-}
-
-dynamo_status dynamo_set_decode_kernel(dynamo_ctx* ctx, int32_t kind) {
-    if (!ctx) return DYNAMO_ERR_NULL;
-    if (kind != DYNAMO_DECODE_TENSOR && kind != DYNAMO_DECODE_STREAM) return DYNAMO_ERR_SHAPE;
-    ctx->decode_kernel = kind;
-    return DYNAMO_OK;
-}
-
 dynamo_status dynamo_set_switch_mode(dynamo_ctx* ctx, int32_t mode) {
     if (!ctx) return DYNAMO_ERR_NULL;
     if (mode != DYNAMO_SWITCH_SELECT && mode != DYNAMO_SWITCH_REQUANT) return DYNAMO_ERR_SHAPE;
@@ -497,6 +499,8 @@ dynamo_status dynamo_pack_experts(dynamo_ctx* ctx, const void* w_gate, const voi
 
     CUDA_TRY(cudaMemsetAsync(ctx->arena, 0, A.total, st));
     CUDA_TRY(cudaMemsetAsync(ctx->ws, 0, ctx->W.total, st));
+    for (size_t g : A.guards) CUDA_TRY(cudaMemsetAsync(ctx->arena + g, GUARD_BYTE, GUARD, st));
+    for (size_t g : ctx->W.guards) CUDA_TRY(cudaMemsetAsync(ctx->ws + g, GUARD_BYTE, GUARD, st));
 
     LayerDev& L = ctx->host_layer;
     std::memset(&L, 0, sizeof(L));
@@ -557,6 +561,7 @@ dynamo_status dynamo_pack_experts(dynamo_ctx* ctx, const void* w_gate, const voi
         if (cudaGetDevice(&dev) == cudaSuccess &&
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
             ctx->n_sms = sms;
+        CUDA_TRY(setup_ffn_tc2(ctx->n_sms, ctx->tc2_clusters));
     }
     ctx->packed = true;
     // install the empty significant sets (sig_pool -> zero tile, sig_chan -> -1)
@@ -675,50 +680,38 @@ static dynamo_status forward_impl(dynamo_ctx* ctx, const void* x, const float* r
     WsDev ws = make_ws(ctx, T);
     const int n = D.n_experts + D.n_shared;
 
-    if (w_router)
-        CUDA_TRY(launch_route_gemm(x, w_router, router_bias, T, D.d_model, D.n_experts, D.top_k, D.renormalize, logits_out,
-                                   ws.topk_idx, ws.topk_w, st));
-    else
-        CUDA_TRY(launch_route(router_logits, T, D.n_experts, D.top_k, D.renormalize, ws.topk_idx, ws.topk_w, st));
-    CUDA_TRY(launch_scan(ws, D.n_experts, D.n_shared, D.top_k, st));
-    CUDA_TRY(launch_gather(L, ws, x, st));
+    const bool fused_front = !w_router && front_fits(T, D.top_k);   // small batch: routing, permutation, gather in one launch
+    if (fused_front) {
+        CUDA_TRY(launch_front(L, ws, x, router_logits, D.n_experts, D.n_shared, D.top_k, D.renormalize, st));
+    } else {
+        if (w_router)
+            CUDA_TRY(launch_route_gemm(x, w_router, router_bias, T, D.d_model, D.n_experts, D.top_k, D.renormalize,
+                                       logits_out, ws.topk_idx, ws.topk_w, st));
+        else
+            CUDA_TRY(launch_route(router_logits, T, D.n_experts, D.top_k, D.renormalize, ws.topk_idx, ws.topk_w, st));
+        CUDA_TRY(launch_scan(ws, D.n_experts, D.n_shared, D.top_k, st));
+        CUDA_TRY(launch_gather(L, ws, x, st));
+    }
     if (ctx->collect_stats) {
         CUDA_TRY(launch_stats(L, ws, x, (float*)(ctx->arena + ctx->A.stats), D.n_experts, st));
         ctx->launches += 1;
     }
     const bool use_tc = ws.tc_min != 0x7fffffff;                  // experts above 32 rows take the tcgen05 path
     const long long split_stride = (long long)ws.Rpad * D.d_model;  // partials of one K split: [Rpad][d]
-    if (ws.fold) {
-        if (ctx->prof_ev[0]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[0], st));
-        CUDA_TRY(launch_ffn_tcd(L, ws, 1, ctx->host_layer.n_rb13, 1, n, split_stride, ctx->n_sms, st));
-        if (ctx->prof_ev[1]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[1], st));
-        CUDA_TRY(launch_ffn_tcd(L, ws, 0, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, ctx->n_sms, st));
-        if (ctx->prof_ev[2]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[2], st));
-        if (ctx->down_active) {
-            CUDA_TRY(launch_down_fix(L, (const DownDev*)ctx->down_arena, ws, D.d_model, st));
-            ctx->launches += 1;
-        }
-        CUDA_TRY(launch_combine(ws, D.d_model, D.top_k, D.n_shared, y, y_dtype == DYNAMO_F32, split_stride, st));
-        ctx->launches += 6;
-        return forward_debug_copies(ctx, ws, T, dbg, st);
-    }
     if (ctx->prof_ev[0]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[0], st));
     const int max_rows = use_tc ? std::min(T, ctx->tc_min_rows) : T;  // rows one expert can have on the streaming path
     CUDA_TRY(launch_ffn_stream(L, ws, 1, ctx->host_layer.n_rb13, 1, n, split_stride, max_rows, ctx->n_sms, st));
-    const bool pair = ctx->prefill_kernel == DYNAMO_PREFILL_PAIR;
-    if (use_tc) CUDA_TRY(pair ? launch_ffn_tc2(L, ws, 1, ctx->host_layer.n_rb13, n, ctx->n_sms, st)
-                              : launch_ffn_tc(L, ws, 1, ctx->host_layer.n_rb13, n, ctx->n_sms, st));
+    if (use_tc) CUDA_TRY(launch_ffn_tc2(L, ws, 1, ctx->host_layer.n_rb13, n, ctx->tc2_clusters[1], st));
     if (ctx->prof_ev[1]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[1], st));
     CUDA_TRY(launch_ffn_stream(L, ws, 0, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, max_rows, ctx->n_sms, st));
-    if (use_tc) CUDA_TRY(pair ? launch_ffn_tc2(L, ws, 0, ctx->host_layer.n_rb2, n, ctx->n_sms, st)
-                              : launch_ffn_tc(L, ws, 0, ctx->host_layer.n_rb2, n, ctx->n_sms, st));
+    if (use_tc) CUDA_TRY(launch_ffn_tc2(L, ws, 0, ctx->host_layer.n_rb2, n, ctx->tc2_clusters[0], st));
     if (ctx->prof_ev[2]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[2], st));
     if (ctx->down_active) {  // significant hidden units: add what their 8-bit columns of W_down change
         CUDA_TRY(launch_down_fix(L, (const DownDev*)ctx->down_arena, ws, D.d_model, st));
         ctx->launches += 1;
     }
     CUDA_TRY(launch_combine(ws, D.d_model, D.top_k, D.n_shared, y, y_dtype == DYNAMO_F32, split_stride, st));
-    ctx->launches += use_tc ? 8 : 6;
+    ctx->launches += (use_tc ? 8 : 6) - (fused_front ? 2 : 0);
     return forward_debug_copies(ctx, ws, T, dbg, st);
 }
 
@@ -918,10 +911,39 @@ dynamo_status dynamo_poll_status(dynamo_ctx* ctx, void* stream) {
     int32_t word = 0;
     CUDA_TRY(cudaMemcpyAsync(&word, ctx->ws + ctx->W.status, 4, cudaMemcpyDeviceToHost, st));
     CUDA_TRY(cudaStreamSynchronize(st));
-    if (word != STATUS_OK) {
-        CUDA_TRY(cudaMemsetAsync(ctx->ws + ctx->W.status, 0, 4, st));
-        return DYNAMO_ERR_TIMEOUT;
-    }
+    if (word == STATUS_OK) return DYNAMO_OK;
+    CUDA_TRY(cudaMemsetAsync(ctx->ws + ctx->W.status, 0, 4, st));
+    if (word & STATUS_TIMEOUT) return DYNAMO_ERR_TIMEOUT;
+    return DYNAMO_ERR_RANGE;
+}
+
+dynamo_status dynamo_debug_expire_wait(dynamo_ctx* ctx, int64_t limit_ns, void* stream) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    if (!ctx->packed) return DYNAMO_ERR_STATE;
+    if (limit_ns < 1000 || limit_ns > 100ll * 1000 * 1000) return DYNAMO_ERR_ARG;
+    CUDA_TRY(launch_expire_wait((int32_t*)(ctx->ws + ctx->W.status), (unsigned long long)limit_ns, (cudaStream_t)stream));
+    ctx->launches += 1;
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_debug_check_guards(dynamo_ctx* ctx, int64_t* n_bad_bytes, void* stream) {
+    if (!ctx || !n_bad_bytes) return DYNAMO_ERR_NULL;
+    if (!ctx->packed) return DYNAMO_ERR_STATE;
+    cudaStream_t st = (cudaStream_t)stream;
+    CUDA_TRY(cudaStreamSynchronize(st));
+    int64_t bad = 0;
+    std::vector<uint8_t> buf(GUARD);
+    auto scan = [&](const uint8_t* base, const std::vector<size_t>& guards) -> cudaError_t {
+        for (size_t g : guards) {
+            cudaError_t err = cudaMemcpy(buf.data(), base + g, GUARD, cudaMemcpyDeviceToHost);
+            if (err != cudaSuccess) return err;
+            for (uint8_t b : buf) bad += b != (uint8_t)GUARD_BYTE;
+        }
+        return cudaSuccess;
+    };
+    CUDA_TRY(scan(ctx->arena, ctx->A.guards));
+    CUDA_TRY(scan(ctx->ws, ctx->W.guards));
+    *n_bad_bytes = bad;
     return DYNAMO_OK;
 }
 

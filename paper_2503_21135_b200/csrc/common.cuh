@@ -18,7 +18,10 @@ constexpr int POOL_TILE_BYTES = 512;   // one cached channel's 8-bit-valued fp16
 constexpr int MAX_EXPERTS = 264;
 constexpr int HI_BITS = 8;
 
-enum : int { STATUS_OK = 0, STATUS_TIMEOUT = 1 };
+// Device status word (bit flags, sticky until dynamo_poll_status clears them).  TIMEOUT: a bounded wait expired,
+// later kernels of the stream start nothing.  RANGE: an activation was clamped to the fp16 operand range (the
+// forward still completes, with the clamped value).
+enum : int { STATUS_OK = 0, STATUS_TIMEOUT = 1, STATUS_RANGE = 2 };
 
 struct ExpertDev {
     const uint8_t* w13;        // packed blocks of the fused gate/up matrix: [n_rb13][n_kc13][blk_bytes]
@@ -77,10 +80,9 @@ struct WsDev {
     uint8_t* xperm;       // [R + pad][d/128][XROW]
     __half* xsig;         // [R + pad][S_pad]
     uint8_t* hbuf;        // [R + pad][f/128][XROW]
-    float* ypart;         // [ksplit][R][d]
+    float* ypart;         // [ksplit][Rpad][d] fp32 rows of the down GEMM, one copy per K split
     int32_t* status;      // device status word
     int32_t T, R, ksplit;
-    int32_t fold;         // 1: every expert goes through the decode tensor-core kernel (operand-tile layout everywhere)
     // Physical rows: every expert's segment starts at a multiple of 8 rows (off_pad), so that the
     // tensor-core path can address activations as 8-row groups.  All row-indexed buffers above use
     // physical rows; Rpad is the host-side bound R + 8 * (E + Es).
@@ -122,6 +124,19 @@ __host__ __device__ __forceinline__ size_t pool_tile_off(int rb, int p, int P_pa
 struct SwitchLayers {
     const LayerDev* layer[64];
 };
+
+// The MMA operands are fp16 and carry a power-of-two pre-scale of at most 2^4, so an activation (an input x or a
+// hidden value h) must satisfy |v| * 16 <= 65504.  Magnitudes above ACT_LIMIT = 4080 (the largest value below
+// 65504 / 16 that both bf16 and fp16 hold exactly; infinities included) are clamped to +-ACT_LIMIT and reported
+// through STATUS_RANGE; NaN passes through.
+constexpr float ACT_LIMIT = 4080.f;
+__device__ __forceinline__ float clamp_act(float v, bool& hit) {
+    if (fabsf(v) > ACT_LIMIT) {
+        hit = true;
+        v = copysignf(ACT_LIMIT, v);
+    }
+    return v;
+}
 
 // ---- PTX helpers -----------------------------------------------------------------------
 
@@ -198,8 +213,11 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
 // the CTA already gave up) it records STATUS_TIMEOUT, raises the CTA-wide poison flag and returns
 // false; callers then leave their loops.
 constexpr unsigned long long WAIT_LIMIT_NS = 1000ull * 1000ull * 1000ull;
+// `where` / `aux` identify the wait: the first waiter of a launch to give up leaves (where, block, thread, aux)
+// in words 8..11 of the status block for the host to read.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* poison,
-                                                  int32_t* status) {
+                                                  int32_t* status, unsigned long long limit_ns = WAIT_LIMIT_NS,
+                                                  int where = 0, int aux = 0) {
     if (mbar_try_wait(bar, parity)) return true;
     // The clock is read only every 1024 failed polls (a poll itself suspends for a while in hardware):
     // reading %globaltimer on every wait that does not pass at once costs far more than the wait.
@@ -212,9 +230,14 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
             const unsigned long long now = globaltimer_ns();
             if (t0 == 0) {
                 t0 = now;
-            } else if (now - t0 > WAIT_LIMIT_NS) {
+            } else if (now - t0 > limit_ns) {
                 *poison = 1;
-                atomicExch(status, STATUS_TIMEOUT);
+                if (atomicCAS(status + 8, 0, where | 0x1000) == 0) {
+                    status[9] = (int)blockIdx.x;
+                    status[10] = (int)threadIdx.x;
+                    status[11] = aux;
+                }
+                atomicOr(status, STATUS_TIMEOUT);
                 return false;
             }
         }
@@ -236,7 +259,7 @@ __device__ __forceinline__ bool mbar_wait_bounded_cluster(uint64_t* bar, uint32_
                 t0 = now;
             } else if (now - t0 > WAIT_LIMIT_NS) {
                 *poison = 1;
-                atomicExch(status, STATUS_TIMEOUT);
+                atomicOr(status, STATUS_TIMEOUT);
                 return false;
             }
         }

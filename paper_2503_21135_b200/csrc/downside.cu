@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(FIX_THREADS) down_fix_kernel(const LayerDev* _
     const int n_e = ws.counts[e];
     const int nrows = min(FIX_ROWS, ws.off_pad[e] + n_e - row0);
     if (cnt <= 0 || nrows <= 0) return;
-    const bool tile_layout = ws.fold || n_e > ws.tc_min;  // which FFN kernel wrote this expert's h
+    const bool tile_layout = n_e > ws.tc_min;  // which FFN kernel wrote this expert's h
     const int bits = L->ex[e].bits, S2 = D2->S2, d = L->d;
     for (int i = threadIdx.x; i < cnt; i += FIX_THREADS) {
         pl[i] = D2->sig_pool[(long long)e * S2 + i];

@@ -88,7 +88,7 @@ __device__ __forceinline__ Item decode_item(const FfnParams& p, const FfnSmem* S
 // items this CTA has finished (parity of the epilogue barrier / h tile).
 template <int BITS, int NT8, bool GATEUP>
 __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uint8_t* stages, uint8_t* htiles,
-                                             const Item& im, int& stage_it, int item_idx) {
+                                             const Item& im, int& stage_it, int item_idx, bool& clamped) {
     constexpr int NS = MAX_STAGES;
     const LayerDev* L = p.L;
     const ExpertDev& ex = L->ex[im.e];
@@ -243,8 +243,9 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     const float g = total[a][j][c], u = total[a][j][2 + c];
-                    const float h = g / (1.f + expf(-g)) * u;
+                    float h = g / (1.f + expf(-g)) * u;
                     const int tok = 8 * j + 2 * tid4 + c;
+                    if (tok < im.nvalid) h = clamp_act(h, clamped);   // columns past the last token hold stale data
                     *reinterpret_cast<__half*>(htile + tok * XROW + (8 * (atom0 + a) + gid) * 2) = __float2half_rn(h);
                 }
         __syncwarp();
@@ -289,13 +290,14 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
 // variants need fewer registers and run three CTAs per SM.
 template <int BITS, bool GATEUP, int MAXNT8>
 __device__ __forceinline__ bool consume_dispatch(const FfnParams& p, FfnSmem* S, uint8_t* stages, uint8_t* htiles,
-                                                 const Item& im, int& stage_it, int item_idx) {
+                                                 const Item& im, int& stage_it, int item_idx, bool& clamped) {
     const int nt8 = (im.nvalid + 7) >> 3;
-    if (MAXNT8 == 1 || nt8 == 1) return consume_item<BITS, 1, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
+    if (MAXNT8 == 1 || nt8 == 1) return consume_item<BITS, 1, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx, clamped);
     if constexpr (MAXNT8 >= 2) {
-        if (MAXNT8 == 2 || nt8 == 2) return consume_item<BITS, 2, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
+        if (MAXNT8 == 2 || nt8 == 2)
+            return consume_item<BITS, 2, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx, clamped);
     }
-    if constexpr (MAXNT8 >= 3) return consume_item<BITS, 3, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx);
+    if constexpr (MAXNT8 >= 3) return consume_item<BITS, 3, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx, clamped);
     return false;
 }
 
@@ -303,7 +305,7 @@ template <bool GATEUP, int MAXNT8>
 __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2) ffn_stream_kernel(const FfnParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     pdl_prologue();
-    if (*p.ws.status != STATUS_OK) return;  // after an expired wait nothing new starts
+    if (*p.ws.status & STATUS_TIMEOUT) return;  // after an expired wait nothing new starts
     const LayerDev* L = p.L;
     FfnSmem* S = reinterpret_cast<FfnSmem*>(smem);
     uint8_t* stages = smem + SMEM_HEADER;
@@ -344,7 +346,9 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
             need = (need + 127) & ~127;
             int pad = 0;
             if (head + need > p.ring_bytes) { pad = p.ring_bytes - head; head = 0; }
-            const int total = need + pad;
+            // a stage that wraps while the write offset is still inside its own footprint needs the whole ring
+            // (its footprint and the skipped tail overlap): then it waits for every earlier stage and takes it all
+            const int total = need + pad < p.ring_bytes ? need + pad : p.ring_bytes;
             while (free_b < total || tail + NS <= it) {
                 const int q = tail % NS;
                 if (!mbar_wait_bounded(&S->empty[q], (tail / NS) & 1, poison, p.ws.status)) return -1;
@@ -453,10 +457,11 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
 
     // ---------------- consumer warps ----------------
     int stage_it = 0, y = 0, item_idx = 0;
+    bool clamped = false;
     (void)G;
     const bool all_static = n_items <= (int)gridDim.x;
     for (;; ++item_idx) {
-        if (all_static && (item_idx > 0 || (int)blockIdx.x >= n_items)) return;
+        if (all_static && (item_idx > 0 || (int)blockIdx.x >= n_items)) break;
         // the next stage opens the next item (or says there is none): its index rides with the stage
         int g = blockIdx.x;  // the first item is dealt statically: decode it while its first stage is in flight
         if (item_idx > 0) {
@@ -464,20 +469,21 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
             if (!mbar_wait_bounded(&S->full[s0], (stage_it / NS) & 1, poison, p.ws.status)) return;
             g = S->first_item[s0];
         }
-        if (g < 0 || g >= n_items) return;
+        if (g < 0 || g >= n_items) break;
         const Item im = decode_item(p, S, g, y);
         bool ok;
         switch (L->ex[im.e].bits) {
-            case 2: ok = consume_dispatch<2, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx); break;
-            case 3: ok = consume_dispatch<3, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx); break;
-            case 4: ok = consume_dispatch<4, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx); break;
-            default: ok = consume_dispatch<8, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx); break;
+            case 2: ok = consume_dispatch<2, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
+            case 3: ok = consume_dispatch<3, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
+            case 4: ok = consume_dispatch<4, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
+            default: ok = consume_dispatch<8, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
         }
         if (!ok) {  // poisoned: the status word says so; keep arriving so that nobody waits on this warp forever
             if (GATEUP && lane == 0) mbar_arrive(&S->done);
             return;
         }
     }
+    if (clamped) atomicOr(p.ws.status, STATUS_RANGE);
 }
 
 template <bool GATEUP, int MAXNT8>

@@ -194,6 +194,10 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
     uint8_t* wring = smem + T2_OFF_STAGE;
     uint8_t* xring = smem + T2_OFF_XRING;
 
+    // After an expired wait nothing new starts.  Both CTAs of a pair read the same word (the preceding kernel has
+    // completed, and every cluster of this persistent grid starts at launch), so they leave together, before any
+    // barrier or tensor memory exists.
+    if (*p.ws.status & STATUS_TIMEOUT) return;
     // Item table (identical in both CTAs of the pair): experts above the row threshold contribute
     // (256-token tiles x row blocks) items.
     for (int i = threadIdx.x; i < p.n_experts; i += T2_THREADS) {
@@ -381,7 +385,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
         const int atom_g = 8 * rank + a_l;   // atom within the 256-row block
         const int gid = lane >> 2, tid4 = lane & 3;
         const uint32_t my_lanes = tbase + ((uint32_t)(32 * q + 16 * asel) << 16);
-        bool ok = true;
+        bool ok = true, clamped = false;
         uint32_t ic = 0;
         for (int g = cluster_id; g < total && ok; g += n_clusters, ++ic) {
             const T2Item w = t2_decode_item<GATEUP>(p, prefix, g, cursor, n_kc, rank);
@@ -451,7 +455,8 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
 #pragma unroll
                             for (int c = 0; c < 2; ++c) {
                                 const float v0 = __uint_as_float(r[4 * j + c]), v1 = __uint_as_float(r[4 * j + 2 + c]);
-                                const float h = __fdividef(v0, 1.f + __expf(-v0)) * v1;
+                                float h = __fdividef(v0, 1.f + __expf(-v0)) * v1;
+                                if (n0 + c < w.n_valid) h = clamp_act(h, clamped);   // columns past the last token: ignored
                                 hs[c] = __half2float(__float2half_rn(h)) * scl;   // exact: scl is a power of two
                             }
                             const int odd = gid & 1;
@@ -483,6 +488,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
             __syncwarp();
             if (lane == 0) mbar_arrive_remote(&B->d_empty, 0);
         }
+        if (clamped) atomicOr(status, STATUS_RANGE);
     }
     // No CTA of the pair may exit (or free tensor memory) while its peer can still reach it.
     tc_fence_before();
@@ -493,47 +499,54 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
     }
 }
 
+// Persistent grid: as many CTA pairs as can be resident at once on the current device (pairs must share a TPC; not
+// every SM may be pairable), so that the static round-robin over clusters has no second wave.  Also raises the
+// kernels' shared-memory limit.  Called once per context at pack time, with the layer's device current.
 template <bool GATEUP>
-static cudaError_t launch_t2_one(const T2Params& p, int n_sms, cudaStream_t st, int* clusters_out) {
+static cudaError_t t2_setup_one(int n_sms, int* clusters_out) {
     cudaError_t err =
         cudaFuncSetAttribute(ffn_tc2_kernel<GATEUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, T2_SMEM_BYTES);
     if (err != cudaSuccess) return err;
-    // Persistent grid: as many CTA pairs as can be resident at once (pairs must share a TPC; not every SM may
-    // be pairable), so that the static round-robin over clusters has no second wave.
-    static int n_clusters[2] = {0, 0};
-    int& nc = n_clusters[GATEUP ? 1 : 0];
-    if (nc == 0) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(n_sms & ~1));
-        cfg.blockDim = dim3(T2_THREADS);
-        cfg.dynamicSmemBytes = T2_SMEM_BYTES;
-        cudaLaunchAttribute at[1];
-        at[0].id = cudaLaunchAttributeClusterDimension;
-        at[0].val.clusterDim.x = 2;
-        at[0].val.clusterDim.y = 1;
-        at[0].val.clusterDim.z = 1;
-        cfg.attrs = at;
-        cfg.numAttrs = 1;
-        int m = 0;
-        err = cudaOccupancyMaxActiveClusters(&m, ffn_tc2_kernel<GATEUP>, &cfg);
-        if (err != cudaSuccess) return err;
-        if (m < 1) return cudaErrorInvalidConfiguration;
-        nc = m < n_sms / 2 ? m : n_sms / 2;
-    }
-    if (clusters_out) *clusters_out = nc;
-    return launch_pdl_cluster(ffn_tc2_kernel<GATEUP>, dim3((unsigned)(2 * nc)), dim3(T2_THREADS), (size_t)T2_SMEM_BYTES, 2u,
-                              st, p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(n_sms & ~1));
+    cfg.blockDim = dim3(T2_THREADS);
+    cfg.dynamicSmemBytes = T2_SMEM_BYTES;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    int m = 0;
+    err = cudaOccupancyMaxActiveClusters(&m, ffn_tc2_kernel<GATEUP>, &cfg);
+    if (err != cudaSuccess) return err;
+    if (m < 1) return cudaErrorInvalidConfiguration;
+    *clusters_out = m < n_sms / 2 ? m : n_sms / 2;
+    return cudaSuccess;
 }
 
-// n_rb: 256-row weight blocks; n_experts: experts in L->order; n_sms: SMs of the device (one CTA each, in pairs).
-cudaError_t launch_ffn_tc2(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int n_experts, int n_sms,
+// clusters_out[0]: down launch, clusters_out[1]: gate/up launch.
+cudaError_t setup_ffn_tc2(int n_sms, int* clusters_out) {
+    cudaError_t err = t2_setup_one<false>(n_sms, &clusters_out[0]);
+    if (err != cudaSuccess) return err;
+    return t2_setup_one<true>(n_sms, &clusters_out[1]);
+}
+
+// n_rb: 256-row weight blocks; n_experts: experts in L->order; n_clusters: CTA pairs of the persistent grid
+// (from setup_ffn_tc2 on this device).
+cudaError_t launch_ffn_tc2(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int n_experts, int n_clusters,
                            cudaStream_t st) {
     T2Params p;
     p.L = L;
     p.ws = ws;
     p.n_rb = n_rb;
     p.n_experts = n_experts;
-    return gateup ? launch_t2_one<true>(p, n_sms, st, nullptr) : launch_t2_one<false>(p, n_sms, st, nullptr);
+    if (n_clusters < 1) return cudaErrorInvalidConfiguration;
+    return gateup ? launch_pdl_cluster(ffn_tc2_kernel<true>, dim3((unsigned)(2 * n_clusters)), dim3(T2_THREADS),
+                                       (size_t)T2_SMEM_BYTES, 2u, st, p)
+                  : launch_pdl_cluster(ffn_tc2_kernel<false>, dim3((unsigned)(2 * n_clusters)), dim3(T2_THREADS),
+                                       (size_t)T2_SMEM_BYTES, 2u, st, p);
 }
 
 }  // namespace dyn

@@ -109,10 +109,6 @@ __global__ void pack_hi_kernel(const __nv_bfloat16* __restrict__ w_gate, const _
 // Re-derive the 8-bit codes (and forward-ready values) of selected cached channels from the bf16
 // originals in the channel cache: channel replacement followed by requantization.
 // list: [n_items] packed (expert << 16 | pool position); grid.x covers rows, grid.y = items, grid.z = mat.
-struct RequantArgs {
-    const LayerDev* layer;
-    const int32_t* items;
-};
 __global__ void requant_from_cache_kernel(const LayerDev* __restrict__ L, const int32_t* __restrict__ items) {
     const int item = items[blockIdx.y];
     const int e = item >> 16, p = item & 0xffff;

@@ -164,8 +164,8 @@ __global__ void __launch_bounds__(1024) scan_kernel(WsDev ws, int E, int Es, int
     const int T = ws.T, n_pairs = T * k;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
     const int kk = k + Es;
-    // work-queue counters of this forward's FFN launches (callers that only route pass no status block)
-    if (ws.status && threadIdx.x < 4) ws.status[4 + threadIdx.x] = 0;
+    // work-queue counters of this forward's streaming launches (callers that only route pass no status block)
+    if (ws.status && threadIdx.x < 2) ws.status[4 + threadIdx.x] = 0;
     const int per_warp = ((n_pairs + 31) / 32 + nwarps - 1) / nwarps * 32;  // whole 32-pair batches per segment
     const int seg_lo = min(n_pairs, warp * per_warp), seg_hi = min(n_pairs, seg_lo + per_warp);
     const unsigned lt = (1u << lane) - 1;
@@ -268,13 +268,9 @@ __global__ void __launch_bounds__(1024) scan_kernel(WsDev ws, int E, int Es, int
 // One CTA per physical row; warp w converts chunks w, w+8, ...  The fp16 activations are stored
 // multiplied by 2^x_scale_exp(bits of the row's expert, k) so that the FFN kernels can use packed codes
 // in place; the per-group sums are of the unscaled fp16 values.
-__global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict__ L, WsDev ws,
-                                                     const __nv_bfloat16* __restrict__ x) {
-    pdl_prologue();
-    const int row = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (row >= ws.off_pad[L->E + L->Es]) return;
-    const int t = ws.row_token[row], e = ws.row_expert[row];
-    const bool tc = ws.fold || ws.counts[e] > ws.tc_min;
+__device__ __forceinline__ void gather_row(const LayerDev* __restrict__ L, const WsDev& ws,
+                                           const __nv_bfloat16* __restrict__ x, int row, int t, int e, bool tc) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (t < 0 && !tc) return;  // padding rows matter only as zero rows of an MMA operand tile
     const int d = L->d;
     const int n_kc = d / KC;
@@ -285,6 +281,7 @@ __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict_
     const float sc0 = __uint_as_float((uint32_t)(127 + x_scale_exp(bits, 4 * lane)) << 23);
     const float sc1 = __uint_as_float((uint32_t)(127 + x_scale_exp(bits, 4 * lane + 2)) << 23);
     const int rg = row >> 3, rr = row & 7;
+    bool clamped = false;
     for (int c = warp; c < n_kc; c += 8) {
         const int k0 = c * KC + lane * 4;
         float v[4] = {0.f, 0.f, 0.f, 0.f};
@@ -293,6 +290,8 @@ __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict_
             const __nv_bfloat162 p0 = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
             const __nv_bfloat162 p1 = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
             v[0] = __low2float(p0); v[1] = __high2float(p0); v[2] = __low2float(p1); v[3] = __high2float(p1);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) v[i] = clamp_act(v[i], clamped);
             if (sw) {
                 const uint32_t mw = mask[k0 >> 5] >> (k0 & 31);
 #pragma unroll
@@ -325,6 +324,7 @@ __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict_
             if ((lane & 15) == 0) *reinterpret_cast<float*>(out + TC_TILE_BYTES + ((lane >> 4) * 8 + rr) * 4) = sum;
         }
     }
+    if (clamped && ws.status) atomicOr(ws.status, STATUS_RANGE);
     // Activations of ALL cached channels of the row's expert, unscaled, zero where the channel is not
     // currently significant: the FFN kernels multiply them with the contiguous 8-bit-valued tiles of the
     // whole cache pool, so a switch only has to flip mask bits.
@@ -338,7 +338,7 @@ __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict_
             float v = 0.f;
             if (j < P) {
                 const int ch = ci[j];
-                if ((mask[ch >> 5] >> (ch & 31)) & 1u) v = __bfloat162float(xr[ch]);
+                if ((mask[ch >> 5] >> (ch & 31)) & 1u) v = clamp_act(__bfloat162float(xr[ch]), clamped);
             }
             *reinterpret_cast<__half*>(xp + xpool_off(pq, row, ws.Rcap) + col * 2) = __float2half_rn(v);
         } else {
@@ -349,7 +349,7 @@ __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict_
             float v = 0.f;
             if (t >= 0 && pj < P) {
                 const int ch = ci[pj];
-                if ((mask[ch >> 5] >> (ch & 31)) & 1u) v = __bfloat162float(xr[ch]);
+                if ((mask[ch >> 5] >> (ch & 31)) & 1u) v = clamp_act(__bfloat162float(xr[ch]), clamped);
             }
             // 8-row operand tile of group pq: [k-octet 4][row 8][8 k] fp16 = 512 B
             *reinterpret_cast<__half*>(xp + xpool_off(pq, 8 * rg, ws.Rcap) + (col >> 3) * 128 + rr * 16 + (col & 7) * 2) =
@@ -358,10 +358,142 @@ __global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict_
     }
 }
 
+__global__ void __launch_bounds__(256) gather_kernel(const LayerDev* __restrict__ L, WsDev ws,
+                                                     const __nv_bfloat16* __restrict__ x) {
+    pdl_prologue();
+    const int row = blockIdx.x;
+    if (row >= ws.off_pad[L->E + L->Es]) return;
+    const int e = ws.row_expert[row];
+    gather_row(L, ws, x, row, ws.row_token[row], e, ws.counts[e] > ws.tc_min);
+}
+
+// Small batches: routing, permutation and gather in ONE launch (three launches cost more than their work when the
+// whole forward takes tens of microseconds).  One CTA per physical row; every CTA repeats the routing and the
+// counting sort of all T * k pairs in shared memory (a few hundred pairs at most), then gathers its own row; CTA 0
+// also writes the routing outputs and the row tables the later kernels read.  Same results as the three kernels.
+constexpr int FRONT_MAX_PAIRS = 128;
+constexpr int FRONT_MAX_TOKENS = 16;   // beyond this the three separate kernels are faster (measured at 32 and 64 tokens)
+__global__ void __launch_bounds__(256) front_kernel(const LayerDev* __restrict__ L, WsDev ws,
+                                                    const __nv_bfloat16* __restrict__ x,
+                                                    const float* __restrict__ logits, int E, int Es, int k, int renorm) {
+    __shared__ int s_idx[FRONT_MAX_PAIRS];
+    __shared__ float s_w[FRONT_MAX_PAIRS];
+    __shared__ int s_rank[FRONT_MAX_PAIRS];
+    __shared__ int s_count[MAX_EXPERTS + 1], s_off[MAX_EXPERTS + 1], s_pad[MAX_EXPERTS + 1];
+    __shared__ int s_row_e, s_row_t;
+    pdl_prologue();
+    const int T = ws.T, n_pairs = T * k, kk = k + Es;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int t = warp; t < T; t += 8) {
+        const float* l = logits + (long long)t * E;
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int e = lane + 32 * i;
+            v[i] = (e < E) ? l[e] : -INFINITY;
+        }
+        topk_softmax_store(v, lane, E, k, renorm, t, s_idx, s_w);
+    }
+    if (threadIdx.x == 0) { s_row_e = -1; s_row_t = -1; }
+    __syncthreads();
+    // counting sort: thread e walks the pairs in order (pair i = t*k + j ascends in t: the stable order)
+    for (int e = threadIdx.x; e < E + Es; e += blockDim.x) {
+        int c = 0;
+        if (e < E) {
+            for (int i = 0; i < n_pairs; ++i)
+                if (s_idx[i] == e) s_rank[i] = c++;
+        } else {
+            c = T;
+        }
+        s_count[e] = c;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int run = 0, run_pad = 0;
+        for (int e0 = 0; e0 < E + Es; e0 += 32) {
+            const int e = e0 + lane;
+            const int c = e < E + Es ? s_count[e] : 0;
+            int v = c, vp = (c + 7) & ~7;
+#pragma unroll
+            for (int dd = 1; dd < 32; dd <<= 1) {
+                const int u = __shfl_up_sync(0xffffffffu, v, dd), up = __shfl_up_sync(0xffffffffu, vp, dd);
+                if (lane >= dd) {
+                    v += u;
+                    vp += up;
+                }
+            }
+            if (e < E + Es) {
+                s_off[e] = run + v - c;
+                s_pad[e] = run_pad + vp - ((c + 7) & ~7);
+            }
+            run += __shfl_sync(0xffffffffu, v, 31);
+            run_pad += __shfl_sync(0xffffffffu, vp, 31);
+        }
+        if (lane == 0) {
+            s_off[E + Es] = run;
+            s_pad[E + Es] = run_pad;
+        }
+    }
+    __syncthreads();
+    const int row = blockIdx.x;
+    // whose row is this: the expert whose padded segment holds it, then the pair of that expert with this rank
+    for (int e = threadIdx.x; e < E + Es; e += blockDim.x)
+        if (row >= s_pad[e] && row < s_pad[e + 1]) s_row_e = e;
+    __syncthreads();
+    const int my_e = s_row_e;
+    if (my_e >= 0) {
+        const int r = row - s_pad[my_e];
+        if (my_e < E) {
+            for (int i = threadIdx.x; i < n_pairs; i += blockDim.x)
+                if (s_idx[i] == my_e && s_rank[i] == r) s_row_t = i / k;
+        } else if (threadIdx.x == 0 && r < T) {
+            s_row_t = r;
+        }
+    }
+    if (blockIdx.x == 0) {
+        if (threadIdx.x < 2) ws.status[4 + threadIdx.x] = 0;   // work-queue counters of the two streaming launches
+        // the outputs and tables of the route and scan kernels
+        for (int i = threadIdx.x; i < n_pairs; i += blockDim.x) {
+            const int e = s_idx[i], r = s_rank[i], t = i / k, j = i - t * k;
+            ws.topk_idx[i] = e;
+            ws.topk_w[i] = s_w[i];
+            ws.perm[s_off[e] + r] = i;
+            ws.pos[t * kk + j] = s_pad[e] + r;
+            ws.row_token[s_pad[e] + r] = t;
+            ws.row_expert[s_pad[e] + r] = e;
+        }
+        for (int e = threadIdx.x; e <= E + Es; e += blockDim.x) {
+            ws.offsets[e] = s_off[e];
+            ws.off_pad[e] = s_pad[e];
+            if (e < E + Es) ws.counts[e] = s_count[e];
+        }
+        for (int e = threadIdx.x; e < E; e += blockDim.x) {
+            const int c = s_count[e], po = s_pad[e];
+            for (int r = c; r < ((c + 7) & ~7); ++r) {
+                ws.row_token[po + r] = -1;
+                ws.row_expert[po + r] = e;
+            }
+        }
+        for (int sx = 0; sx < Es; ++sx) {
+            const int po = s_pad[E + sx];
+            const int padded = (T + 7) & ~7;
+            for (int t = threadIdx.x; t < padded; t += blockDim.x) {
+                if (t < T) ws.pos[t * kk + k + sx] = po + t;
+                ws.row_token[po + t] = t < T ? t : -1;
+                ws.row_expert[po + t] = E + sx;
+            }
+        }
+    }
+    __syncthreads();
+    if (my_e < 0) return;
+    gather_row(L, ws, x, row, s_row_t, my_e, s_count[my_e] > ws.tc_min);
+}
+
 // grid (T, ceil(d / 1024)): each thread owns four output columns of one token.
 __global__ void __launch_bounds__(256) combine_kernel(WsDev ws, int d, int k, int Es, void* __restrict__ y,
                                                       int y_f32, long long split_stride) {
     pdl_prologue();
+    if (*ws.status & STATUS_TIMEOUT) return;  // the FFN kernels started nothing: leave y alone
     const int t = blockIdx.x;
     const int kk = k + Es;
     const int c = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
@@ -371,7 +503,7 @@ __global__ void __launch_bounds__(256) combine_kernel(WsDev ws, int d, int k, in
         const int r = ws.pos[t * kk + j];
         const float w = (j < k) ? ws.topk_w[t * k + j] : 1.0f;
         float s[4] = {0.f, 0.f, 0.f, 0.f};
-        const int ns = (!ws.fold && ws.counts[ws.row_expert[r]] > ws.tc_min) ? 1 : ws.ksplit;  // the tensor-core path does not split K
+        const int ns = (ws.counts[ws.row_expert[r]] > ws.tc_min) ? 1 : ws.ksplit;  // the tensor-core path does not split K
         for (int sp = 0; sp < ns; ++sp) {
             const float4 v = *reinterpret_cast<const float4*>(ws.ypart + sp * split_stride + (long long)r * d + c);
             s[0] += v.x; s[1] += v.y; s[2] += v.z; s[3] += v.w;
@@ -406,6 +538,12 @@ cudaError_t launch_scan(const WsDev& ws, int E, int Es, int k, cudaStream_t st) 
 }
 cudaError_t launch_gather(const LayerDev* L, const WsDev& ws, const void* x, cudaStream_t st) {
     return launch_pdl(gather_kernel, dim3((unsigned)ws.Rpad), dim3(256), 0, st, L, ws, (const __nv_bfloat16*)x);
+}
+bool front_fits(int T, int k) { return T <= FRONT_MAX_TOKENS && T * k <= FRONT_MAX_PAIRS; }
+cudaError_t launch_front(const LayerDev* L, const WsDev& ws, const void* x, const float* logits, int E, int Es, int k,
+                         int renorm, cudaStream_t st) {
+    return launch_pdl(front_kernel, dim3((unsigned)ws.Rpad), dim3(256), 0, st, L, ws, (const __nv_bfloat16*)x, logits, E,
+                      Es, k, renorm);
 }
 cudaError_t launch_combine(const WsDev& ws, int d, int k, int Es, void* y, int y_f32, long long split_stride,
                            cudaStream_t st) {

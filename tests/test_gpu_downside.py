@@ -89,21 +89,15 @@ def test_forward_with_down_side_sets(lay, T):
     assert torch.equal(_forward(lay, T, step=T)[0], y0)
 
 
-def test_other_kernels_and_all_cached_units(lay):
+def test_all_cached_units_on_both_kernels(lay):
     gpu = lay["gpu"]
     sets = [p[:S2] for p in lay["pool_d"]]
     _install(lay, sets)
     try:
-        gpu.set_prefill_kernel(binding.PREFILL_SINGLE)
-        y, ref = _forward(lay, 200, step=3)
-        assert rel_err(y.cpu().numpy(), ref) <= TOL
-        gpu.set_prefill_kernel(binding.PREFILL_PAIR)
-        gpu.set_decode_kernel(binding.DECODE_TENSOR)
-        y, ref = _forward(lay, 33, step=4)
-        assert rel_err(y.cpu().numpy(), ref) <= TOL
+        for T, step in ((200, 3), (33, 4)):     # tcgen05 kernel for the popular experts; streaming kernel only
+            y, ref = _forward(lay, T, step=step)
+            assert rel_err(y.cpu().numpy(), ref) <= TOL
     finally:
-        gpu.set_prefill_kernel(binding.PREFILL_PAIR)
-        gpu.set_decode_kernel(binding.DECODE_STREAM)
         _install(lay, [np.array([], np.int32)] * CFG.n_experts)
 
 

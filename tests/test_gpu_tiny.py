@@ -84,7 +84,6 @@ def test_tensor_core_and_streaming_kernels_agree_with_the_oracle(tiny, T):
     every expert on the streaming kernel (large experts as 32-token chunks)."""
     gpu = tiny["gpu"]
     out = {}
-    gpu.set_decode_kernel(binding.DECODE_STREAM)
     try:
         for rows in (8, 0):
             gpu.set_tc_min_rows(rows)
@@ -102,23 +101,6 @@ def test_tensor_core_and_streaming_kernels_agree_with_the_oracle(tiny, T):
         launches.append(gpu.kernel_launches() - n0)
     gpu.set_tc_min_rows(32)
     assert launches[0] - launches[1] == 2, launches
-
-
-@pytest.mark.parametrize("T", [1, 7, 16, 17, 33, 64])
-def test_decode_tensor_and_streaming_kernels_agree_with_the_oracle(tiny, T):
-    """Small batches through the streaming kernel (default) and through the decode tensor-core kernel."""
-    gpu = tiny["gpu"]
-    out = {}
-    try:
-        for kind in (binding.DECODE_TENSOR, binding.DECODE_STREAM):
-            gpu.set_decode_kernel(kind)
-            y, _, ref, _, _ = _forward_both(tiny, T, tiny["sets"], step=500 + T)
-            assert rel_err(y, ref["y"]) <= TOL, (kind, rel_err(y, ref["y"]))
-            out[kind] = y
-    finally:
-        gpu.set_decode_kernel(binding.DECODE_STREAM)
-    diff = np.max(np.abs(out[binding.DECODE_TENSOR] - out[binding.DECODE_STREAM]))
-    assert diff <= 1e-3 * np.sqrt(np.mean(out[binding.DECODE_STREAM].astype(np.float64) ** 2)), diff
 
 
 def test_empty_sets_and_bf16_output(tiny):
@@ -265,7 +247,7 @@ def test_forward_can_be_captured_in_a_cuda_graph(tiny):
     with torch.cuda.graph(graph):
         gpu.forward(xs, ls, binding.F32, y=ys)
     per_forward = gpu.kernel_launches() - n0
-    assert per_forward == 6
+    assert per_forward in (4, 6)       # small batches fuse routing, permutation and gather into one launch
     xs.copy_(x)
     ls.copy_(lg)
     for _ in range(3):

@@ -455,31 +455,41 @@ def test_router_scores_match_library_matmul_and_closed_forms():
 
 # ---- runtime selection of the significant channels ---------------------------------------------
 
-def test_channel_stats_closed_forms_and_order():
+def test_channel_stats_closed_forms():
     rng = np.random.default_rng(5)
     T, d, E, k, P = 40, 64, 4, 2, 8
     idx = np.stack([rng.permutation(E)[:k] for _ in range(T)]).astype(np.int32)
     pool = np.stack([np.sort(rng.permutation(d)[:P]) for _ in range(E)]).astype(np.int32)
-    # |x| = 1 everywhere: the statistic is the number of tokens routed to the expert (exact in float32)
+    # |x| = 1 everywhere: the statistic is the number of tokens routed to the expert
     ones = bf16_bits(np.where(rng.random((T, d)) < 0.5, 1.0, -1.0))
-    s = oracle.channel_stats_update(np.zeros((E, P), np.float32), ones, idx, pool)
-    assert np.array_equal(s, np.tile(np.bincount(idx.ravel(), minlength=E).astype(np.float32)[:, None], (1, P)))
+    s = oracle.channel_stats_update(np.zeros((E, P)), ones, idx, pool)
+    assert s.dtype == np.float64
+    assert np.array_equal(s, np.tile(np.bincount(idx.ravel(), minlength=E).astype(np.float64)[:, None], (1, P)))
     # x zero outside one channel: only that channel (where cached) accumulates, by the routed tokens' |x|
     xz = np.zeros((T, d))
-    xz[:, pool[1, 3]] = rng.integers(1, 5, size=T)                    # small integers: sums exact
-    s = oracle.channel_stats_update(np.zeros((E, P), np.float32), bf16_bits(xz), idx, pool)
+    xz[:, pool[1, 3]] = rng.integers(1, 5, size=T) * np.where(rng.random(T) < 0.5, 1.0, -1.0)
+    s = oracle.channel_stats_update(np.zeros((E, P)), bf16_bits(xz), idx, pool)
     for e in range(E):
         toks = (idx == e).any(axis=1)
-        expect = np.where(pool[e] == pool[1, 3], xz[toks, pool[1, 3]].sum(), 0.0)
-        assert np.array_equal(s[e], expect.astype(np.float32))
-    # two updates add: running total = first + second (integers: no rounding)
+        expect = np.where(pool[e] == pool[1, 3], np.abs(xz[toks, pool[1, 3]]).sum(), 0.0)
+        assert np.array_equal(s[e], expect)
+    # two updates add: running total = first + second
     s2 = oracle.channel_stats_update(s, bf16_bits(xz), idx, pool)
     assert np.array_equal(s2, 2 * s)
-    # float32, token-ascending order: 2^24 + 1 + 1 stays 2^24 in that order (a float64 or reordered sum would not)
+    # exact sums: 2^24 + 1 + 1 keeps both ones, and the result does not depend on the order of the tokens
     big = np.zeros((3, d))
-    big[0, pool[0, 0]], big[1, pool[0, 0]], big[2, pool[0, 0]] = 2.0 ** 24, 1.0, 1.0
-    s3 = oracle.channel_stats_update(np.zeros((E, P), np.float32), bf16_bits(big), np.zeros((3, 1), np.int32), pool)
-    assert s3[0, 0] == np.float32(2.0 ** 24)
+    big[0, pool[0, 0]], big[1, pool[0, 0]], big[2, pool[0, 0]] = 2.0 ** 24, 1.0, -1.0
+    routed = np.zeros((3, 1), np.int32)
+    s3 = oracle.channel_stats_update(np.zeros((E, P)), bf16_bits(big), routed, pool)
+    assert s3[0, 0] == 2.0 ** 24 + 2
+    assert np.array_equal(oracle.channel_stats_update(np.zeros((E, P)), bf16_bits(big[::-1].copy()), routed, pool), s3)
+    # random data against a library routine: a masked matrix product of |x|
+    xr = bf16_bits(rng.standard_normal((T, d)))
+    xa = np.abs((xr.astype(np.uint32) << 16).view(np.float32)).astype(np.float64)
+    s4 = oracle.channel_stats_update(np.zeros((E, P)), xr, idx, pool)
+    member = np.stack([(idx == e).any(axis=1) for e in range(E)]).astype(np.float64)       # [E, T]
+    full = member @ xa                                                                     # [E, d]
+    assert np.allclose(s4, np.take_along_axis(full, pool.astype(np.int64), axis=1), rtol=1e-13, atol=0)
 
 
 def test_select_significant_rank_rule():

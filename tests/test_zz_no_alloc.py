@@ -1,14 +1,15 @@
-"""The allocation-free routing entry point against the regular forward's routing outputs.
+"""The allocation-free routing entry point against the regular forward's routing outputs and the CPU oracle.
 
 Callers that may not allocate device memory (stream capture in progress, framework plugins with a
 fixed buffer set, real-time loops) use dynamo_route_permute_static; it must give exactly what
-dynamo_moe_forward reports for the same logits, call after call, although all calls share one
-scratch array inside the library.  This file sorts last so that a stop-at-first-failure run has
+dynamo_moe_forward reports for the same logits, and exactly the oracle's top-k and permutation, call
+after call, although all calls share one scratch array inside the library.  This file sorts last so that a stop-at-first-failure run has
 already executed every other test."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from helpers import make_gpu_layer, make_inputs
 from paper_2503_21135_b200 import binding
 from paper_2503_21135_b200 import workloads as wl
@@ -45,6 +46,13 @@ def test_static_route_matches_forward_twice_in_a_row():
         assert torch.equal(off, dbg["offsets"])
         assert torch.equal(perm, dbg["perm"])
         assert float((w - dbg["w"]).abs().max()) <= 1e-6
+        # and directly against the oracle: indices, offsets and permutation bit-exact, weights to 1e-6
+        ref_idx, ref_w = oracle.route(lg.cpu().numpy(), CFG.top_k)
+        ref_off, ref_perm = oracle.permute(ref_idx, CFG.n_experts)
+        assert np.array_equal(idx.cpu().numpy(), ref_idx)
+        assert np.array_equal(off.cpu().numpy(), ref_off)
+        assert np.array_equal(perm.cpu().numpy(), ref_perm)
+        assert float(np.max(np.abs(w.cpu().numpy() - ref_w))) <= 1e-6
 
 
 def test_static_route_limits():
