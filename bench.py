@@ -7,8 +7,11 @@ through one MoE layer, via the C-ABI call ``dynamo_moe_forward``.  Steps rotate 
 independently generated layers so that the packed weights of a step always come from HBM (the
 rotating set is far larger than L2).
 
-Prints ONE JSON line (see README / DESIGN for the keys).  ``--impl reference`` times the CPU oracle
-instead (a deliberately plain float64 program; it is a reported baseline, not a target).
+Prints ONE JSON line.  The default run (decode workload) carries the whole metric: the headline is decode at
+T = 64; ``extra`` holds T = 1, 8, 32, 64 with the HBM roofline of the gate/up launch each, the prefill workload
+(T = 4096) with its tensor roofline, and ``switch`` the runtime channel switch on a 16-layer stack.
+``--impl reference`` times the CPU oracle instead (a deliberately plain float64 program; it is a reported
+baseline, not a target).
 """
 from __future__ import annotations
 
@@ -98,13 +101,37 @@ class ClockSampler:
         return out
 
 
-def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None, down_side=0):
+def device_layer_weights(cfg, layer, device):
+    """The weight recipe of workloads.expert_weights (N(0, 0.02^2), each routed expert's outlier input channels
+    x20 in W_gate and W_up, rounded to bf16) drawn on the device: a 1.4-billion-weight layer takes the host cores
+    ten seconds and the GPU a few milliseconds, and the timed runs need many layers.  Same distribution, other
+    draws than the host recipe, which stays the one the parity tests and the CPU baseline use."""
+    g = torch.Generator(device=device)
+    g.manual_seed(wl.BASE_SEED * 1000 + cfg.config_id * 100 + layer)
+    n, d, f = cfg.n_total, cfg.d_model, cfg.d_ff
+    out = []
+    for shape, outliers in (((n, f, d), True), ((n, f, d), True), ((n, d, f), False)):
+        w = torch.empty(shape, dtype=torch.float32, device=device)
+        w.normal_(0.0, 0.02, generator=g)
+        if outliers:
+            for e in range(cfg.n_experts):
+                cols = torch.from_numpy(wl.outlier_channels(cfg, layer, e).astype(np.int64)).to(device)
+                w[e][:, cols] *= 20.0
+        out.append(w.to(torch.bfloat16))
+        del w
+    return tuple(out)
+
+
+def build_layers(cfg, n_layers, max_tokens, device, tc_min_rows=None, down_side=0, host_recipe=False):
     """Generate, upload and pack ``n_layers`` independent layers; they share one workspace."""
     from paper_2503_21135_b200 import binding
 
     layers, meta, ws = [], [], None
     for l in range(n_layers):
-        wg, wu, wd = wl.layer_weights(cfg, l, threads=min(16, os.cpu_count() or 8))
+        if host_recipe:
+            wg, wu, wd = wl.layer_weights(cfg, l, threads=min(16, os.cpu_count() or 8))
+        else:
+            wg, wu, wd = device_layer_weights(cfg, l, device)
         bits = wl.bits_assignment(cfg, l)
         pool = wl.cache_pool(cfg, l)
         sets = wl.initial_sig_sets(cfg, pool, l)
@@ -183,6 +210,101 @@ def job_throughput(tokens_per_rank, world, ms_per_step):
     return world * tokens_per_rank / (ms_per_step / 1e3)
 
 
+def time_workload(cfg, layers, meta, T, steps, warmup, rank, world, device, barrier, hbm_peak, tensor_peak, peak_kind,
+                  want_clocks=True):
+    """Time `steps` forwards of T tokens rotating over `layers`; returns a result dict with throughput, the live
+    per-launch times of the two FFN launches and the roofline block of the dominant (gate/up) launch."""
+    from paper_2503_21135_b200 import binding
+
+    n_layers = len(layers)
+    xs = [wl.activations(cfg, T, l, step=0).to(device) for l in range(n_layers)]
+    lgs_cpu = [wl.router_logits(cfg, T, l, step=0) for l in range(n_layers)]
+    lgs = [t.to(device) for t in lgs_cpu]
+    ys = [torch.empty((T, cfg.d_model), dtype=torch.float32, device=device) for _ in range(n_layers)]
+
+    def step(i):
+        l = i % n_layers
+        layers[l].forward(xs[l], lgs[l], binding.F32, y=ys[l])
+
+    sampler = ClockSampler(torch.cuda.current_device()) if want_clocks and rank == 0 else None
+    if sampler:
+        sampler.start()
+        t_end = time.time() + 0.6        # keep the GPU under load while the sampler comes up
+        while time.time() < t_end:
+            for i in range(20):
+                step(i)
+            torch.cuda.synchronize()
+    for i in range(max(warmup, 3)):
+        step(i)
+    torch.cuda.synchronize()
+    l0 = sum(l.kernel_launches() for l in layers)
+    ms = time_steps(step, steps, barrier)
+    launches = sum(l.kernel_launches() for l in layers) - l0
+    gu_ms, dn_ms = kernel_times(layers, step, max(steps, 50))
+    clocks = sampler.stop() if sampler else None
+    for l in layers:
+        assert l.poll_status() == 0, "device status word set (expired wait or clamped activation)"
+    (ms_step,) = slowest_rank([ms / steps], world, device)
+    res = {"tokens": T, "steps": steps, "ms_per_step": ms_step, "tokens_per_s": job_throughput(T, world, ms_step),
+           "gpu_launches": launches, "gateup_ms": gu_ms, "down_ms": dn_ms, "clocks": clocks}
+    d, f, G = cfg.d_model, cfg.d_ff, cfg.group_size
+    pick = [i % n_layers for i in range(steps)]
+    if T >= 512:
+        # prefill-sized: the gate/up tcgen05 launch is bound by the tensor cores.  Algorithmic flops of the launch =
+        # 2 * 2 * d * f per (token, expert) row + 2 * 2 * f * |S_e| for rows of switchable experts.
+        fl = []
+        for i in range(n_layers):
+            idx = torch.topk(lgs_cpu[i], cfg.top_k, dim=1).indices.flatten()
+            cnt = torch.bincount(idx, minlength=cfg.n_experts).tolist() + [T] * cfg.n_shared
+            fl.append(sum(c * (4 * d * f + (4 * f * len(meta[i]["sets"][e])
+                                            if e < cfg.n_experts and int(meta[i]["bits"][e]) < 8 else 0))
+                          for e, c in enumerate(cnt)))
+        gu_flops = float(np.mean([fl[i] for i in pick]))
+        achieved = gu_flops / (gu_ms / 1e3) / 1e12
+        burst = measured_burst()
+        res["roofline"] = {"bound": "tensor", "achieved": achieved, "peak": tensor_peak, "unit": "TFLOP/s",
+                           "frac": achieved / tensor_peak, "traffic": None,
+                           "peak_kind": peak_kind + " (sustained fp16/bf16 cuBLAS; the kernel runs inside a long step)",
+                           "frac_of_burst_peak": achieved / burst if burst else None, "burst_peak": burst,
+                           "frac_of_nominal_2250": achieved / 2250.0,
+                           "kernel": "ffn_tc2_kernel<gate/up> (+ streaming kernel for experts of <= 32 rows)",
+                           "algorithmic_flops_per_launch": gu_flops, "avg_launch_ms": gu_ms,
+                           "down_launch": {"achieved": gu_flops / 2 / (dn_ms / 1e3) / 1e12, "avg_launch_ms": dn_ms},
+                           "whole_step": {"achieved": 1.5 * gu_flops / (ms_step / 1e3) / 1e12,
+                                          "frac": 1.5 * gu_flops / (ms_step / 1e3) / 1e12 / tensor_peak,
+                                          "frac_of_nominal_2250": 1.5 * gu_flops / (ms_step / 1e3) / 1e12 / 2250.0}}
+    else:
+        # decode-sized: HBM-bound on the packed bytes (+ significant tiles) of the experts a step activates
+        gu_b, dn_b = [], []
+        for i in range(n_layers):
+            act = active_experts(cfg, lgs_cpu[i])
+            tot = sum(layers[i].stream_bytes(e) for e in act)
+            dn = sum(d * f * int(meta[i]["bits"][e]) // 8 + d * f // G * 4 for e in act)
+            gu_b.append(tot - dn)
+            dn_b.append(dn)
+        gu_bytes = float(np.mean([gu_b[i] for i in pick]))
+        dn_bytes = float(np.mean([dn_b[i] for i in pick]))
+        achieved = gu_bytes / (gu_ms / 1e3) / 1e9
+        step_gbs = (gu_bytes + dn_bytes) / (ms_step / 1e3) / 1e9
+        res["roofline"] = {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+                           "frac": achieved / hbm_peak, "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, T)),
+                           "peak_kind": peak_kind, "frac_of_nominal_8000": achieved / 8000.0,
+                           "kernel": "ffn_stream_kernel<gate/up>",
+                           "algorithmic_bytes_per_launch": gu_bytes, "avg_launch_ms": gu_ms,
+                           "down_launch": {"achieved": dn_bytes / (dn_ms / 1e3) / 1e9, "avg_launch_ms": dn_ms},
+                           "whole_step": {"achieved": step_gbs, "frac": step_gbs / hbm_peak,
+                                          "frac_of_nominal_8000": step_gbs / 8000.0}}
+    return res, (xs, lgs_cpu)
+
+
+def measured_burst():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(p))["bf16_tflops"])
+    except Exception:
+        return None
+
+
 def run_ours(args, rank, world, device):
     from paper_2503_21135_b200 import binding, build
 
@@ -190,72 +312,36 @@ def run_ours(args, rank, world, device):
     binding.load()
     cfg = wl.CONFIGS[args.workload]
     T = args.tokens
-    n_layers = args.layers
     hbm_peak, tensor_peak, peak_kind = measured_peaks()
+    full = args.workload == "decode" and not args.single   # the default run: the whole metric on one line
 
     def barrier():
         if world > 1:
             torch.distributed.barrier()
 
+    n_layers = args.layers if not full else max(args.layers, 16 if not args.no_switch else args.layers)
     layers, meta = build_layers(cfg, n_layers, max(T, max(cfg.tokens)), device, args.tc_min_rows, args.down_side)
-    sweep_T = sorted(set([T] + (list(cfg.tokens) if args.sweep else [])))
-    results = {}
+    rot = layers[:args.layers], meta[:args.layers]     # the layers a timed run rotates over (weights from HBM)
+    common = dict(rank=rank, world=world, device=device, barrier=barrier, hbm_peak=hbm_peak, tensor_peak=tensor_peak,
+                  peak_kind=peak_kind)
+    head, _ = time_workload(cfg, rot[0], rot[1], T, args.steps, args.warmup, **common)
+    extra = {}
+    sweep_T = [t for t in cfg.tokens if t != T] if (full or args.sweep) else []
     for Tcur in sweep_T:
-        xs = [wl.activations(cfg, Tcur, l, step=0).to(device) for l in range(n_layers)]
-        lgs_cpu = [wl.router_logits(cfg, Tcur, l, step=0) for l in range(n_layers)]
-        lgs = [t.to(device) for t in lgs_cpu]
-        ys = [torch.empty((Tcur, cfg.d_model), dtype=torch.float32, device=device) for _ in range(n_layers)]
-
-        def step(i):
-            l = i % n_layers
-            layers[l].forward(xs[l], lgs[l], binding.F32, y=ys[l])
-
-        main = Tcur == T
-        sampler = ClockSampler(torch.cuda.current_device()) if main and rank == 0 else None
-        if sampler:
-            sampler.start()
-            t_end = time.time() + 0.6        # keep the GPU under load while the sampler comes up
-            while time.time() < t_end:
-                for i in range(50):
-                    step(i)
-                torch.cuda.synchronize()
-        for i in range(max(args.warmup, 3)):
-            step(i)
-        torch.cuda.synchronize()
-        l0 = sum(l.kernel_launches() for l in layers)
-        ms = time_steps(step, args.steps, barrier)
-        launches = sum(l.kernel_launches() for l in layers) - l0
-        clocks = sampler.stop() if sampler else None
-        for l in layers:
-            assert l.poll_status() == 0, "device-side wait expired"
-        # algorithmic HBM bytes: packed blocks (+ significant tiles) of the experts a step activates
-        gu_bytes, dn_bytes = [], []
-        d, f, G = cfg.d_model, cfg.d_ff, cfg.group_size
-        for i in range(n_layers):
-            act = active_experts(cfg, lgs_cpu[i])
-            tot = sum(layers[i].stream_bytes(e) for e in act)
-            dn = sum(d * f * int(meta[i]["bits"][e]) // 8 + d * f // G * 4 for e in act)
-            gu_bytes.append(tot - dn)
-            dn_bytes.append(dn)
-        pick = [i % n_layers for i in range(args.steps)]
-        res = dict(ms_total=ms, ms_per_step=ms / args.steps, launches=launches, clocks=clocks,
-                   gu_bytes=float(np.mean([gu_bytes[i] for i in pick])),
-                   dn_bytes=float(np.mean([dn_bytes[i] for i in pick])))
-        res["bytes_per_step"] = res["gu_bytes"] + res["dn_bytes"]
-        res["gu_ms"], res["dn_ms"] = kernel_times(layers, step, args.steps)
-        results[Tcur] = res
+        extra[str(Tcur)], _ = time_workload(cfg, rot[0], rot[1], Tcur, max(args.steps, 200), args.warmup, **common)
+    extra[str(T)] = head
 
     router = None
     if args.router:
         # the same step with the router GEMM + top-k fused in front (scores from synthetic router weights, so the
         # routing differs from the logits-input run above: compare times at token counts where every expert is active)
-        wr = [wl.router_weights(cfg, l) for l in range(n_layers)]
-        wrd = [(w.to(device), b.to(device)) for w, b in wr]
-        xs = [wl.activations(cfg, T, l, step=0).to(device) for l in range(n_layers)]
+        nl = len(rot[0])
+        wrd = [tuple(t.to(device) for t in wl.router_weights(cfg, l)) for l in range(nl)]
+        xs = [wl.activations(cfg, T, l, step=0).to(device) for l in range(nl)]
 
         def step_router(i):
-            l = i % n_layers
-            layers[l].forward_router(xs[l], wrd[l][0], wrd[l][1], binding.F32)
+            l = i % nl
+            rot[0][l].forward_router(xs[l], wrd[l][0], wrd[l][1], binding.F32)
 
         for i in range(max(args.warmup, 3)):
             step_router(i)
@@ -263,77 +349,55 @@ def run_ours(args, rank, world, device):
         router = {"ms_per_step_with_router_gemm": ms_r / args.steps, "tokens_per_s": world * T / (ms_r / args.steps / 1e3)}
 
     # end-to-end through the host-buffer entry point (pinned host memory, copies inside the timed region)
-    xh = [wl.activations(cfg, T, l, step=0).pin_memory() for l in range(n_layers)]
-    lh = [wl.router_logits(cfg, T, l, step=0).pin_memory() for l in range(n_layers)]
-    yh = [torch.empty((T, cfg.d_model), dtype=torch.float32).pin_memory() for _ in range(n_layers)]
+    nl = len(rot[0])
+    xh = [wl.activations(cfg, T, l, step=0).pin_memory() for l in range(nl)]
+    lh = [wl.router_logits(cfg, T, l, step=0).pin_memory() for l in range(nl)]
+    yh = [torch.empty((T, cfg.d_model), dtype=torch.float32).pin_memory() for _ in range(nl)]
 
     def step_host(i):
-        l = i % n_layers
-        layers[l].forward_host(xh[l], lh[l], yh[l], binding.F32)
+        l = i % nl
+        rot[0][l].forward_host(xh[l], lh[l], yh[l], binding.F32)
 
     for i in range(3):
         step_host(i)
     ms_e2e = time_steps(step_host, args.steps, barrier)
-
-    r = results[T]
-    ms_step = r["ms_per_step"]
-    ms_step, ms_e2e = slowest_rank([ms_step, ms_e2e], world, device)
-    value = job_throughput(T, world, ms_step)
-    e2e_value = job_throughput(T, world, ms_e2e / args.steps)
+    (ms_e2e,) = slowest_rank([ms_e2e / args.steps], world, device)
 
     out = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f16 (integer codes x fp16 activations, fp32 accumulate)", "data": "synthetic",
+        "metric": METRIC, "value": head["tokens_per_s"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": "f16 (integer codes x fp16 activations, fp32 accumulate)", "data": "synthetic (weights drawn on the device from the recipe's distribution, activations and logits from the seeded host recipe)",
         "config": {"workload": f"{cfg.name}: d_model={cfg.d_model} d_ff={cfg.d_ff} E={cfg.n_experts} top{cfg.top_k} "
                                f"G={cfg.group_size} S={cfg.max_sig} T={T}",
-                   "tokens": T, "layers_rotated": n_layers, "l2": "inputs larger than L2 (rotating layer arenas)",
+                   "tokens": T, "layers_rotated": len(rot[0]), "l2": "inputs larger than L2 (rotating layer arenas)",
                    "parallelism": "replicas only" if world > 1 else "single gpu",
                    **({"down_side_significant": args.down_side} if args.down_side else {})},
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": T * cfg.d_model * 2 + T * cfg.n_experts * 4,
+        "e2e": {"value": job_throughput(T, world, ms_e2e), "unit": UNIT,
+                "h2d_bytes_per_step": T * cfg.d_model * 2 + T * cfg.n_experts * 4,
                 "d2h_bytes_per_step": T * cfg.d_model * 4},
-        "gpu_launches": r["launches"],
-        "clocks": r["clocks"],
+        "gpu_launches": head["gpu_launches"],
+        "clocks": head["clocks"],
+        "roofline": head["roofline"],
     }
-    if T >= 512:
-        # prefill-sized: the gate/up tcgen05 launch is bound by the tensor cores.  Algorithmic flops of the
-        # launch = 2 * 2 * d * f per (token, expert) row + 2 * 2 * f * |S_e| for rows of switchable experts.
-        d, f = cfg.d_model, cfg.d_ff
-        fl = []
-        for i in range(n_layers):
-            idx = torch.topk(wl.router_logits(cfg, T, i, 0), cfg.top_k, dim=1).indices.flatten()
-            cnt = torch.bincount(idx, minlength=cfg.n_experts).tolist() + [T] * cfg.n_shared
-            fl.append(sum(c * (4 * d * f + (4 * f * len(meta[i]["sets"][e])
-                                            if e < cfg.n_experts and int(meta[i]["bits"][e]) < 8 else 0))
-                          for e, c in enumerate(cnt)))
-        gu_flops = float(np.mean([fl[i % n_layers] for i in range(args.steps)]))
-        achieved = gu_flops / (r["gu_ms"] / 1e3) / 1e12
-        out["roofline"] = {"bound": "tensor", "achieved": achieved, "peak": tensor_peak, "unit": "TFLOP/s",
-                           "frac": achieved / tensor_peak, "traffic": None, "peak_kind": peak_kind + " (sustained fp16/bf16)",
-                           "kernel": "ffn_tc2_kernel<gate/up> (+ streaming kernel for experts of <= 32 rows)",
-                           "algorithmic_flops_per_launch": gu_flops, "avg_launch_ms": r["gu_ms"],
-                           "down_launch": {"achieved": gu_flops / 2 / (r["dn_ms"] / 1e3) / 1e12, "avg_launch_ms": r["dn_ms"]},
-                           "whole_step_tflops": 1.5 * gu_flops / (ms_step / 1e3) / 1e12}
-    # roofline of the dominant kernel: the gate/up launch of ffn_stream_kernel (2/3 of the packed bytes)
-    achieved = r["gu_bytes"] / (r["gu_ms"] / 1e3) / 1e9
-    if T < 512:
-      out["roofline"] = {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
-                       "frac": achieved / hbm_peak, "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, T)),
-                       "peak_kind": peak_kind,
-                       "kernel": "ffn_stream_kernel<gate/up>",
-                       "algorithmic_bytes_per_launch": r["gu_bytes"], "avg_launch_ms": r["gu_ms"],
-                       "down_launch": {"achieved": r["dn_bytes"] / (r["dn_ms"] / 1e3) / 1e9, "avg_launch_ms": r["dn_ms"]},
-                       "whole_step": {"achieved": r["bytes_per_step"] / (ms_step / 1e3) / 1e9,
-                                      "frac": r["bytes_per_step"] / (ms_step / 1e3) / 1e9 / hbm_peak}}
     if router is not None:
         out["router"] = router
-    out["extra"] = {str(t): {"tokens_per_s": world * t / (v["ms_per_step"] / 1e3), "ms_per_step": v["ms_per_step"],
-                             "gateup_ms": v["gu_ms"], "down_ms": v["dn_ms"],
-                             "step_gbs": v["bytes_per_step"] / (v["ms_per_step"] / 1e3) / 1e9,
-                             "step_frac_of_peak": v["bytes_per_step"] / (v["ms_per_step"] / 1e3) / 1e9 / hbm_peak}
-                    for t, v in results.items()}
     if cfg.n_experts == 8 and cfg.d_model == 4096 and not args.no_switch:
         out["switch"] = measure_switch(layers, meta, cfg, device)
+    del layers, rot
+    torch.cuda.empty_cache()
+    if full and not args.no_prefill:
+        # the prefill half of the metric: config 3 (4096 tokens, Zipf-skewed router), its own layers and roofline
+        pcfg = wl.CONFIGS["prefill"]
+        pT = max(pcfg.tokens)
+        players, pmeta = build_layers(pcfg, 2, pT, device, args.tc_min_rows, 0)
+        pres, _ = time_workload(pcfg, players, pmeta, pT, max(args.steps, 50), args.warmup, **common)
+        pres["workload"] = (f"{pcfg.name}: d_model={pcfg.d_model} d_ff={pcfg.d_ff} E={pcfg.n_experts} top{pcfg.top_k} "
+                            f"G={pcfg.group_size} S={pcfg.max_sig} T={pT}, 2 layers rotated")
+        extra[f"prefill_{pT}"] = pres
+        del players
+        torch.cuda.empty_cache()
+    out["extra"] = extra
     if rank == 0 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(cfg, T, args.cpu_tokens)
     return out
@@ -473,12 +537,24 @@ def run_reference(args, rank, world):
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
 
+def spawn_ranks(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: run the same command line as N local ranks under torchrun."""
+    import socket
+
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=50)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "replica-selftest"])
     ap.add_argument("--workload", default="decode", choices=list(wl.CONFIGS))
     ap.add_argument("--tokens", type=int, default=None, help="default: the workload's largest token count")
     ap.add_argument("--layers", type=int, default=None,
@@ -491,6 +567,10 @@ def main():
     ap.add_argument("--down-side", type=int, default=0,
                     help="also serve this many significant hidden units per expert at 8-bit on the d_ff side (W_down)")
     ap.add_argument("--sweep", action="store_true", help="also time the workload's other token counts")
+    ap.add_argument("--single", action="store_true",
+                    help="only the headline token count (the default decode run also reports T = 1, 8, 32, the prefill "
+                         "workload and the 16-layer switch stack)")
+    ap.add_argument("--no-prefill", action="store_true", help="skip the prefill entry of the default run")
     ap.add_argument("--cpu-tokens", type=int, default=16, help="tokens in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -499,6 +579,9 @@ def main():
     if args.layers is None:
         args.layers = wl.CONFIGS[args.workload].n_layers if args.workload == "switch" else (2 if args.tokens >= 512 else 4)
 
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        # no launcher around us: start one rank per GPU ourselves (independent replicas; see slowest_rank)
+        raise SystemExit(spawn_ranks(args.gpus))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -506,6 +589,16 @@ def main():
         out = run_reference(args, rank, world)
         if out is not None:
             print(json.dumps(out), flush=True)
+        return
+    if args.impl == "replica-selftest":
+        # the N > 1 plumbing alone (rendezvous, MAX-reduction of timings, one line from rank 0), on gloo without a GPU
+        torch.distributed.init_process_group("gloo")
+        got = slowest_rank([1.0 + rank], world, torch.device("cpu"))
+        torch.distributed.barrier()
+        torch.distributed.destroy_process_group()
+        if rank == 0:
+            print(json.dumps({"impl": "replica-selftest", "n_gpus": world, "ms_per_step": got[0],
+                              "value": job_throughput(1, world, got[0])}), flush=True)
         return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")

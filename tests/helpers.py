@@ -34,16 +34,18 @@ def rel_err(y_gpu: np.ndarray, y_ref: np.ndarray) -> float:
     return float(np.max(np.abs(y_gpu.astype(np.float64) - y_ref))) / max(rms, 1e-300)
 
 
-def stratified_tokens(idx: np.ndarray, E: int, n: int, seed: int = 0) -> np.ndarray:
-    """A seeded subset of tokens that touches every expert: all tokens of the two least-loaded
-    experts (capped) plus a uniform sample."""
+def stratified_tokens(idx: np.ndarray, E: int, n: int, seed: int = 0, all_of_two_least: bool = False) -> np.ndarray:
+    """A seeded subset of at least n tokens that touches every expert: the tokens of the two least-loaded experts
+    (all of them if asked, else capped at n/4 each), one token of every other expert, then a uniform sample."""
     T = idx.shape[0]
     rng = np.random.default_rng(seed)
     counts = np.bincount(idx.ravel(), minlength=E)
     chosen = set()
     order = np.argsort(counts, kind="stable")
     for e in order[:2]:
-        toks = np.flatnonzero((idx == e).any(axis=1))[: max(1, n // 4)]
+        toks = np.flatnonzero((idx == e).any(axis=1))
+        if not all_of_two_least:
+            toks = toks[: max(1, n // 4)]
         chosen.update(int(t) for t in toks)
     for e in range(E):
         toks = np.flatnonzero((idx == e).any(axis=1))

@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 TOL = 1e-2
 
 
-def _check_forward(cfg, gpu, ora, T, n_sample, step=0, layer=0):
+def _check_forward(cfg, gpu, ora, T, n_sample, step=0, layer=0, all_of_two_least=False):
     x, lg = wl.activations(cfg, T, layer, step), wl.router_logits(cfg, T, layer, step)
     y, dbg = gpu.forward(x.cuda(), lg.cuda(), binding.F32, debug=True)
     torch.cuda.synchronize()
@@ -26,7 +26,8 @@ def _check_forward(cfg, gpu, ora, T, n_sample, step=0, layer=0):
     assert np.array_equal(dbg["offsets"].cpu().numpy(), offsets)
     assert np.array_equal(dbg["perm"].cpu().numpy(), perm)
     assert np.max(np.abs(dbg["w"].cpu().numpy().astype(np.float64) - w)) <= 1e-6
-    toks = stratified_tokens(idx, cfg.n_experts, n_sample, seed=step) if n_sample < T else np.arange(T, dtype=np.int32)
+    toks = (stratified_tokens(idx, cfg.n_experts, n_sample, seed=step, all_of_two_least=all_of_two_least)
+            if n_sample < T else np.arange(T, dtype=np.int32))
     ref = ora.forward(oracle.as_u16(x), lg.numpy(), tokens=toks)["y"][toks]
     got = y.cpu().numpy()[toks]
     assert np.all(np.isfinite(y.cpu().numpy()))
@@ -49,7 +50,9 @@ def test_prefill_config():
         q, s, m = gpu.export_codes(e, binding.MAT_DOWN)
         assert torch.equal(q.cpu(), torch.from_numpy(ora.base[e][2].q))
         assert np.array_equal(s.cpu().numpy().view(np.uint16), ora.base[e][2].s)
-    idx = _check_forward(cfg, gpu, ora, 4096, 96)
+    # the bench size: at least 512 stratified tokens, among them ALL tokens of the two least-loaded experts (every
+    # row of their token tiles, ragged last tile included, is compared with the oracle)
+    idx = _check_forward(cfg, gpu, ora, 4096, 512, all_of_two_least=True)
     counts = np.bincount(idx.ravel(), minlength=8)
     assert counts[7] == counts.max() and counts[7] > 2 * counts[0]        # Zipf skew: expert 7 most loaded
     # a ragged token count that leaves partial 32-token chunks in every expert
@@ -130,33 +133,69 @@ def test_finegrained_config_with_shared_experts():
 
 
 def test_switch_stress_stack():
+    """Config 5: the 16-layer stack at decode batch 16.  Every layer is compared with the oracle at step 0 and after
+    the first switch event (one call for the whole stack); layers 0 and 1 also after the next two events.  The
+    oracle of a layer is built, asked for its reference outputs and dropped (sixteen of them do not fit the host)."""
     cfg = wl.CONFIGS["switch"]
-    n_layers, T = 3, 16
-    gpus, oras, pools, cur, ws = [], [], [], [], None
+    n_layers, T = cfg.n_layers, 16
+    assert n_layers == 16
+    gpus, pools, cur, ws = [], [], [], None
+    refs = {}          # (layer, event index or -1) -> dict(idx, perm, y)
+    keep = {}          # oracle layers of the two layers followed further
+    new_sets = []
     for l in range(n_layers):
         wg, wu, wd, bits, pool, sets = make_inputs(cfg, layer=l)
         g = make_gpu_layer(cfg, wg, wu, wd, bits, pool, max_tokens=T, workspace=ws)
         ws = g.workspace
         gpus.append(g)
-        oras.append(make_oracle_layer(cfg, wg, wu, wd, bits))
         pools.append(pool)
         cur.append(sets)
+        new = wl.switch_event(cfg, pool, sets, l, 0)
+        for e in range(cfg.n_experts):
+            assert len(np.setdiff1d(new[e], sets[e])) == 16               # 25 % of 64 swapped
+        new_sets.append(new)
+        need = set()
+        for step in (0, 8):
+            idx, _ = oracle.route(wl.router_logits(cfg, T, l, step).numpy(), cfg.top_k)
+            need |= set(int(e) for e in idx.ravel())
+        ora = make_oracle_layer(cfg, wg, wu, wd, bits, experts=sorted(need) if l >= 2 else None)
+        for tag, s_, step in ((-1, sets, 0), (0, new, 8)):
+            ora.set_channel_switch(s_)
+            x, lg = wl.activations(cfg, T, l, step), wl.router_logits(cfg, T, l, step)
+            refs[(l, tag)] = ora.forward(oracle.as_u16(x), lg.numpy())
+        if l < 2:
+            keep[l] = ora
+        del ora, wg, wu, wd
+
+    def check(l, tag, step):
+        x, lg = wl.activations(cfg, T, l, step), wl.router_logits(cfg, T, l, step)
+        y, dbg = gpus[l].forward(x.cuda(), lg.cuda(), binding.F32, debug=True)
+        torch.cuda.synchronize()
+        assert gpus[l].poll_status() == 0
+        ref = refs[(l, tag)]
+        assert np.array_equal(dbg["idx"].cpu().numpy(), ref["idx"])
+        assert np.array_equal(dbg["perm"].cpu().numpy(), ref["perm"])
+        err = rel_err(y.cpu().numpy(), ref["y"])
+        assert err <= TOL, (l, tag, err)
+
     binding.set_channel_switch_many(gpus, cur)
     for l in range(n_layers):
-        oras[l].set_channel_switch(cur[l])
-    step = 0
-    for event in range(3):
-        for l in range(n_layers):
-            _check_forward(cfg, gpus[l], oras[l], T, T, step=step, layer=l)
+        check(l, -1, 0)
+    binding.set_channel_switch_many(gpus, new_sets)                        # one upload + one launch for the stack
+    cur = new_sets
+    for l in range(n_layers):
+        check(l, 0, 8)
+    step = 8
+    for event in (1, 2):
         step += 8
         new = [wl.switch_event(cfg, pools[l], cur[l], l, event) for l in range(n_layers)]
-        for l in range(n_layers):
-            for e in range(cfg.n_experts):
-                assert len(np.setdiff1d(new[l][e], cur[l][e])) == 16       # 25 % of 64 swapped
-        binding.set_channel_switch_many(gpus, new)                         # one upload + one launch for the stack
-        for l in range(n_layers):
-            oras[l].set_channel_switch(new[l])
+        binding.set_channel_switch_many(gpus, new)
         cur = new
+        for l in (0, 1):
+            keep[l].set_channel_switch(new[l])
+            x, lg = wl.activations(cfg, T, l, step), wl.router_logits(cfg, T, l, step)
+            refs[(l, event)] = keep[l].forward(oracle.as_u16(x), lg.numpy())
+            check(l, event, step)
     # all-or-nothing: one bad layer rejects the whole event and nothing changes
     x, lg = wl.activations(cfg, T, 0, 99).cuda(), wl.router_logits(cfg, T, 0, 99).cuda()
     y0 = gpus[0].forward(x, lg).clone()
