@@ -323,7 +323,7 @@ def run_ours(args, rank, world, device):
     layers, meta = build_layers(cfg, n_layers, max(T, max(cfg.tokens)), device, args.tc_min_rows, args.down_side)
     rot = layers[:args.layers], meta[:args.layers]     # the layers a timed run rotates over (weights from HBM)
     common = dict(rank=rank, world=world, device=device, barrier=barrier, hbm_peak=hbm_peak, tensor_peak=tensor_peak,
-                  peak_kind=peak_kind)
+                  peak_kind=peak_kind, want_clocks=not args.no_clocks)
     head, _ = time_workload(cfg, rot[0], rot[1], T, args.steps, args.warmup, **common)
     extra = {}
     sweep_T = [t for t in cfg.tokens if t != T] if (full or args.sweep) else []
@@ -571,6 +571,8 @@ def main():
                     help="only the headline token count (the default decode run also reports T = 1, 8, 32, the prefill "
                          "workload and the 16-layer switch stack)")
     ap.add_argument("--no-prefill", action="store_true", help="skip the prefill entry of the default run")
+    ap.add_argument("--no-clocks", action="store_true",
+                    help="no clock sampling (and none of the load that precedes it): for short runs under a profiler")
     ap.add_argument("--cpu-tokens", type=int, default=16, help="tokens in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

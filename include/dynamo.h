@@ -261,7 +261,9 @@ dynamo_status dynamo_select_significant(dynamo_ctx* ctx, int32_t n_select, int32
  *   originals (the channel cache) and differences.  All sets start empty.  Synchronises the stream.
  * dynamo_set_channel_switch_down: installs the sets (the state depends only on the last call).
  *   sig_idx : host int32 [E, max_sig_down], sig_cnt : host int32 [E], 0 <= cnt <= max_sig_down
- *   8-bit experts are validated but keep the empty set.  Synchronises the stream.
+ *   8-bit experts are validated but keep the empty set.  Stream-ordered like dynamo_set_channel_switch: a switch
+ *   enqueued between two forwards takes effect exactly between them (the tables travel by three small copies from
+ *   pageable host memory, which the CUDA runtime stages before the call returns).
  * dynamo_export_codes with DYNAMO_MAT_DOWN and DYNAMO_CODES_HI_POOL / HI_ACTIVE returns the 8-bit codes of the
  * cached / significant hidden units (0 elsewhere) and the 8-bit parameters, shaped like the base export.
  * dynamo_set_channel_precision does not reach this side: it stays at 8 bits.

@@ -861,7 +861,8 @@ dynamo_status dynamo_set_channel_switch_down(dynamo_ctx* ctx, const int32_t* sig
     CUDA_TRY(cudaMemcpyAsync(base + ctx->DA.sig_chan, chan.data(), chan.size() * 4, cudaMemcpyHostToDevice, st));
     CUDA_TRY(cudaMemcpyAsync(base + ctx->DA.sig_pool, pool.data(), pool.size() * 4, cudaMemcpyHostToDevice, st));
     CUDA_TRY(cudaMemcpyAsync(base + ctx->DA.sig_cnt, cnts.data(), cnts.size() * 4, cudaMemcpyHostToDevice, st));
-    CUDA_TRY(cudaStreamSynchronize(st));  // pageable staging: the vectors die with this call
+    // (copies from pageable memory return once the source has been staged, so the vectors may die with this call;
+    // the tables change in stream order, between the forwards enqueued before and after)
     ctx->sig_down = lists;
     ctx->down_active = 0;
     for (int e = 0; e < E; ++e) ctx->down_active += cnts[e] > 0 ? 1 : 0;

@@ -101,6 +101,32 @@ def test_all_cached_units_on_both_kernels(lay):
         _install(lay, [np.array([], np.int32)] * CFG.n_experts)
 
 
+def test_switch_enqueued_between_two_forwards_takes_effect_between_them(lay):
+    """No host synchronisation anywhere in the sequence forward, switch, forward, switch back, forward: every
+    forward must see exactly the set installed before it in stream order."""
+    gpu = lay["gpu"]
+    T = 24
+    x, lg = wl.activations(CFG, T, step=41).cuda(), wl.router_logits(CFG, T, step=41).cuda()
+    empty = [np.array([], np.int32)] * CFG.n_experts
+    sets = wl.sig_sets_down(CFG, lay["pool_d"], S2)
+    gpu.set_channel_switch_down(empty)
+    y_empty = gpu.forward(x, lg, binding.F32).clone()
+    gpu.set_channel_switch_down(sets)
+    y_sets = gpu.forward(x, lg, binding.F32).clone()
+    torch.cuda.synchronize()
+    assert not torch.equal(y_empty, y_sets)
+    outs = [torch.empty_like(y_empty) for _ in range(3)]
+    gpu.set_channel_switch_down(empty)
+    gpu.forward(x, lg, binding.F32, y=outs[0])
+    gpu.set_channel_switch_down(sets)          # enqueued behind the first forward, ahead of the second
+    gpu.forward(x, lg, binding.F32, y=outs[1])
+    gpu.set_channel_switch_down(empty)
+    gpu.forward(x, lg, binding.F32, y=outs[2])
+    torch.cuda.synchronize()
+    assert torch.equal(outs[0], y_empty) and torch.equal(outs[1], y_sets) and torch.equal(outs[2], y_empty)
+    lay["ora"].set_channel_switch_down(empty)
+
+
 def test_down_side_errors_leave_state(lay):
     gpu, pool_d = lay["gpu"], lay["pool_d"]
     E = CFG.n_experts
