@@ -84,6 +84,15 @@ __device__ __forceinline__ Item decode_item(const FfnParams& p, const FfnSmem* S
     return it;
 }
 
+// m16n8k16 with a zero C operand: d = a * b
+__device__ __forceinline__ void mma16816_z(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%10,%10,%10,%10};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
+}
+
 // Consumer side of one work item.  `stage_it` is the CTA-wide ring position, `item_idx` the number of
 // items this CTA has finished (parity of the epilogue barrier / h tile).
 template <int BITS, int NT8, bool GATEUP>
@@ -127,13 +136,7 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
         const uint8_t* st = stages + S->off[s];
         const uint8_t* xs = st + blk_bytes;
         const uint32_t* prm = reinterpret_cast<const uint32_t*>(st + code_bytes);
-        float accg[APW][NT8][4];
-#pragma unroll
-        for (int a = 0; a < APW; ++a)
-#pragma unroll
-            for (int j = 0; j < NT8; ++j)
-#pragma unroll
-                for (int c = 0; c < 4; ++c) accg[a][j][c] = 0.f;
+        float accg[APW][NT8][4];   // the first MMA of a quantization group starts from a zero C operand
 
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -141,8 +144,9 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
 #pragma unroll
             for (int a = 0; a < APW; ++a) load_codes<BITS>(cd[a], st + (atom0 + a) * atom_bytes(BITS), lane, half);
 
-            auto step = [&](auto S4c) {
+            auto step = [&](auto S4c, auto firstc) {
                 constexpr int S4 = decltype(S4c)::value;
+                constexpr bool FIRST = decltype(firstc)::value;
                 const int sidx = half * 4 + S4;
                 uint32_t b0[NT8], b1[NT8];
 #pragma unroll
@@ -157,13 +161,17 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
                     uint32_t af[4];
                     expand<BITS, S4>(cd[a], af);
 #pragma unroll
-                    for (int j = 0; j < NT8; ++j) mma16816(accg[a][j], af, b0[j], b1[j]);
+                    for (int j = 0; j < NT8; ++j) {
+                        if constexpr (FIRST) mma16816_z(accg[a][j], af, b0[j], b1[j]);
+                        else mma16816(accg[a][j], af, b0[j], b1[j]);
+                    }
                 }
             };
-            step(std::integral_constant<int, 0>{});
-            step(std::integral_constant<int, 1>{});
-            step(std::integral_constant<int, 2>{});
-            step(std::integral_constant<int, 3>{});
+            if (G == 64 || half == 0) step(std::integral_constant<int, 0>{}, std::true_type{});
+            else step(std::integral_constant<int, 0>{}, std::false_type{});
+            step(std::integral_constant<int, 1>{}, std::false_type{});
+            step(std::integral_constant<int, 2>{}, std::false_type{});
+            step(std::integral_constant<int, 3>{}, std::false_type{});
 
             if (G == 64 || half == 1) {
                 // fold the group: total += (s * unscale) * acc + m * sum(x); two FMAs per element
@@ -189,8 +197,6 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
                         total[a][j][1] = fmaf(s0, accg[a][j][1], fmaf(f0.y, xs1[j], total[a][j][1]));
                         total[a][j][2] = fmaf(s1, accg[a][j][2], fmaf(f1.y, xs0[j], total[a][j][2]));
                         total[a][j][3] = fmaf(s1, accg[a][j][3], fmaf(f1.y, xs1[j], total[a][j][3]));
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) accg[a][j][c] = 0.f;
                     }
                 }
             }
