@@ -95,7 +95,7 @@ enum { DYNAMO_SWITCH_SELECT = 0,   /* switch = re-point the active list at codes
 dynamo_status dynamo_create(const dynamo_layer_desc* desc, dynamo_ctx** out);
 dynamo_status dynamo_destroy(dynamo_ctx* ctx);
 
-/* Bytes the caller must provide for the packed weights arena (persistent layer state:
+/* (Utility call: the paper has no counterpart.)  Bytes the caller must provide for the packed weights arena (persistent layer state:
  * packed codes, params, channel cache, 8-bit pool, switch tables) and for the workspace
  * (scratch of pack and forward; may be shared by several layers whose calls are ordered on
  * one stream).  bits: host int32 [E + E_s], routed experts in {2,3,4,8}, shared experts 8.
@@ -177,7 +177,7 @@ dynamo_status dynamo_moe_forward_router(dynamo_ctx* ctx, const void* x, const vo
 dynamo_status dynamo_moe_forward_host(dynamo_ctx* ctx, const void* x_host, const float* logits_host, int32_t T,
                                       void* y_host, int32_t y_dtype, void* stream);
 
-/* Unpack the stored representation back to logical codes, for parity checks.
+/* (Utility call: the paper has no counterpart.)  Unpack the stored representation back to logical codes, for parity checks.
  *   q : dev uint8 [out, in] logical codes (row-major, out = f for gate/up, d for down)
  *   scale_f16, zero_f16 : dev uint16 [out, in/G] fp16 bit patterns
  * which = DYNAMO_CODES_*; the HI variants exist for gate/up of routed experts with bits < 8
@@ -185,9 +185,12 @@ dynamo_status dynamo_moe_forward_host(dynamo_ctx* ctx, const void* x_host, const
 dynamo_status dynamo_export_codes(dynamo_ctx* ctx, int32_t expert, int32_t matrix, uint8_t* q,
                                   uint16_t* scale_f16, uint16_t* zero_f16, int32_t which, void* stream);
 
-/* Algorithmic HBM bytes of one expert as the forward streams it: packed base codes + base params
- * of the three matrices, plus (bits < 8) the 8-bit-valued fp16 tiles of its currently significant
- * channels.  Host only (uses the sets last installed). */
+/* Algorithmic HBM bytes of one expert per forward (the roofline numerator; the paper has no counterpart): packed
+ * base codes + base params of the three matrices, plus (bits < 8) the fp16 tiles of its currently SIGNIFICANT
+ * channels, 2 * d_ff * |S_e| * 2 bytes.  What the kernels actually read is a little more: they stream the tiles of
+ * the whole cache pool (cache_size channels, zero activations for the ones that are not significant), so that a
+ * switch never moves a tile; the difference counts against the achieved fraction as traffic beyond the algorithmic
+ * bytes.  Host only (uses the sets last installed). */
 dynamo_status dynamo_expert_stream_bytes(dynamo_ctx* ctx, int32_t expert, size_t* bytes);
 
 /* Synchronises the stream, reads the device status word and clears it.  (Utility call: the paper has no
@@ -228,10 +231,11 @@ dynamo_status dynamo_set_channel_precision(dynamo_ctx* ctx, const int32_t* hi_bi
  *
  * dynamo_set_stats_collection(on): while on, every forward also accumulates, per routed expert e and cached
  *   channel c, A[e][c] += sum over the tokens routed to e in that forward of |x[t][c]| -- in fp32, tokens in
- *   ascending order inside a forward and ONE addition of the forward's sum to the running total, so the statistics
- *   are reproducible bit for bit (they decide an integer selection).  One extra kernel per forward.  The paper
- *   leaves the statistic open ("significance of channel weights ... corresponding to the tokens"); the activation
- *   mass of the input channel is the reading taken here.
+ *   ascending order inside a forward and ONE addition of the forward's sum to the running total, so two runs give
+ *   the same bits (the statistics decide an integer selection); against exact sums they carry the fp32
+ *   accumulation error n * 2^-24 * A.  One extra kernel per forward.  The paper defines the significance of a
+ *   channel only loosely (Section III-A, and Section IV-A's definition of expert significance built on it); the
+ *   activation mass of the input channel is the reading taken here.
  * dynamo_get_channel_stats: copies A to stats_out, DEVICE fp32 [E, P] (column j = cached channel cache_idx[e][j]).
  * dynamo_select_significant: per expert with base bits < 8 the n_select (<= max_sig, <= P) cached channels with
  *   the largest A, ties -> lower channel index, become the significant set (slot order = rank order); 8-bit
