@@ -3,7 +3,7 @@
  *
  * One MoE layer = one context.  The layer's routed-expert SwiGLU FFN runs over
  * expert-level mixed-precision weights (each expert bit-packed at its own base
- * bit-width, group-wise fp16 scale / fp16 zero) combined with the channel-level
+ * bit-width of 2, 3, 4, 6 or 8 bits, group-wise fp16 scale / fp16 zero) combined with the channel-level
  * dynamic switch: a runtime-selected set of significant input channels per expert
  * is served at 8-bit precision from the channel cache while the rest stay at the
  * expert's base precision.
@@ -45,7 +45,7 @@ typedef enum {
     DYNAMO_OK = 0,
     DYNAMO_ERR_NULL = 1,            /* a required pointer is NULL */
     DYNAMO_ERR_SHAPE = 2,           /* a dimension violates the shape rules above */
-    DYNAMO_ERR_BITS = 3,            /* a bit-width is not one of 2, 3, 4, 8 (shared experts: 8) */
+    DYNAMO_ERR_BITS = 3,            /* a bit-width is not one of 2, 3, 4, 6, 8 (shared experts: 8) */
     DYNAMO_ERR_ALIGN = 4,           /* an arena is not 256-byte aligned, or x / y / w_router not 16-byte aligned */
     DYNAMO_ERR_ARENA_TOO_SMALL = 5, /* weights arena or workspace smaller than dynamo_arena_bytes says */
     DYNAMO_ERR_INDEX_RANGE = 6,     /* a channel index is outside [0, d_model) or a count outside [0, S] */
@@ -98,7 +98,8 @@ dynamo_status dynamo_destroy(dynamo_ctx* ctx);
 /* (Utility call: the paper has no counterpart.)  Bytes the caller must provide for the packed weights arena (persistent layer state:
  * packed codes, params, channel cache, 8-bit pool, switch tables) and for the workspace
  * (scratch of pack and forward; may be shared by several layers whose calls are ordered on
- * one stream).  bits: host int32 [E + E_s], routed experts in {2,3,4,8}, shared experts 8.
+ * one stream).  bits: host int32 [E + E_s], routed experts in {2,3,4,6,8} (the paper's INT2/4/6/8 plus 3),
+ * shared experts 8.
  * Host only. */
 dynamo_status dynamo_arena_bytes(const dynamo_layer_desc* desc, const int32_t* bits,
                                  size_t* weights_bytes, size_t* workspace_bytes);

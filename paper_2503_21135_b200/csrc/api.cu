@@ -135,7 +135,7 @@ dynamo_status check_bits(const dynamo_layer_desc& D, const int32_t* bits) {
         const int b = bits[e];
         if (e >= D.n_experts) {
             if (b != 8) return DYNAMO_ERR_BITS;
-        } else if (b != 2 && b != 3 && b != 4 && b != 8) {
+        } else if (b != 2 && b != 3 && b != 4 && b != 6 && b != 8) {
             return DYNAMO_ERR_BITS;
         }
     }

@@ -19,6 +19,14 @@ template <>
 struct Codes<4> { uint32_t w[4], ws[4]; };
 template <>
 struct Codes<8> { uint32_t w[8]; };
+template <>
+struct Codes<6> { uint32_t w[4], ws[4], t[2][4]; };  // low-nibble words and their >> 8; four copies of the high-bit words
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+    return r;
+}
 
 __device__ __forceinline__ uint32_t rotr32(uint32_t v, int n) { return __funnelshift_r(v, v, n); }
 
@@ -34,6 +42,21 @@ __device__ __forceinline__ void load_codes(Codes<BITS>& c, const uint8_t* atom, 
         const uint4 v1 = *reinterpret_cast<const uint4*>(atom + (2 * half + 1) * 512 + lane * 16);
         c.w[0] = v0.x; c.w[1] = v0.y; c.w[2] = v0.z; c.w[3] = v0.w;
         c.w[4] = v1.x; c.w[5] = v1.y; c.w[6] = v1.z; c.w[7] = v1.w;
+    } else if constexpr (BITS == 6) {
+        const uint4 v = *reinterpret_cast<const uint4*>(atom + half * 512 + lane * 16);
+        c.w[0] = v.x; c.w[1] = v.y; c.w[2] = v.z; c.w[3] = v.w;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) c.ws[i] = c.w[i] >> 8;
+        const uint2 hb = *reinterpret_cast<const uint2*>(atom + 1024 + lane * 16 + half * 8);
+        const uint32_t hw[2] = {hb.x, hb.y};
+#pragma unroll
+        for (int rh = 0; rh < 2; ++rh) {
+            const uint32_t sw = prmt(hw[rh], 0u, 0x2301u);   // bytes of each 16-bit half swapped
+            c.t[rh][0] = hw[rh];
+            c.t[rh][1] = hw[rh] >> 2;
+            c.t[rh][2] = sw;
+            c.t[rh][3] = sw >> 2;
+        }
     } else if constexpr (BITS == 2) {
         const uint2 v = *reinterpret_cast<const uint2*>(atom + lane * 16 + half * 8);
         c.w[0] = v.x; c.w[1] = v.y;
@@ -48,12 +71,6 @@ __device__ __forceinline__ void load_codes(Codes<BITS>& c, const uint8_t* atom, 
     }
 }
 
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t r;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
-    return r;
-}
-
 // A-fragment registers of step S4 (0..3) of the loaded half chunk: fp16 pairs q * 2^(o-24).
 template <int BITS, int S4, uint32_t MAGIC = 0u>
 __device__ __forceinline__ void expand(const Codes<BITS>& c, uint32_t (&a)[4]) {
@@ -66,6 +83,17 @@ __device__ __forceinline__ void expand(const Codes<BITS>& c, uint32_t (&a)[4]) {
             for (int rh = 0; rh < 2; ++rh) {
                 const uint32_t src = (phi < 2) ? c.w[rh * 2 + jj] : c.ws[rh * 2 + jj];
                 a[rh + 2 * h] = (src & (0x000F000Fu << (4 * (phi & 1)))) | MAGIC;
+            }
+        }
+    } else if constexpr (BITS == 6) {
+        constexpr int jj = S4 >> 1;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int phi = 2 * (S4 & 1) + h;
+#pragma unroll
+            for (int rh = 0; rh < 2; ++rh) {
+                const uint32_t lo = (phi < 2) ? c.w[rh * 2 + jj] : c.ws[rh * 2 + jj];
+                a[rh + 2 * h] = (lo & (0x000F000Fu << (4 * h))) | ((c.t[rh][S4] & (0x00300030u << (4 * h))) | MAGIC);
             }
         }
     } else if constexpr (BITS == 8) {
@@ -102,7 +130,7 @@ __device__ __forceinline__ void expand(const Codes<BITS>& c, uint32_t (&a)[4]) {
 template <int BITS>
 __host__ __device__ constexpr int code_offset(int s4, int h) {
     const int phi = 2 * s4 + h;
-    return BITS == 2 ? (phi <= 4 ? 2 * phi : 2 * phi - 10) : BITS == 3 ? 2 * (phi & 3) : BITS == 4 ? 4 * h : 0;
+    return BITS == 2 ? (phi <= 4 ? 2 * phi : 2 * phi - 10) : BITS == 3 ? 2 * (phi & 3) : (BITS == 4 || BITS == 6) ? 4 * h : 0;
 }
 
 }  // namespace dyn

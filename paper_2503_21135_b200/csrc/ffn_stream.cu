@@ -483,6 +483,7 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
             case 2: ok = consume_dispatch<2, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
             case 3: ok = consume_dispatch<3, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
             case 4: ok = consume_dispatch<4, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
+            case 6: ok = consume_dispatch<6, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
             default: ok = consume_dispatch<8, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
         }
         if (!ok) {  // poisoned: the status word says so; keep arriving so that nobody waits on this warp forever

@@ -126,9 +126,9 @@ __device__ __forceinline__ void t2_dequant_half(const uint8_t* st, uint32_t a_co
                                                 uint64_t* release) {
     const int gid = lane >> 2;
     const int ngrp = KC / G;
-    constexpr int BIAS = BITS == 2 ? 4 : (BITS == 3 ? 3 : (BITS == 4 ? 2 : 0));
-    constexpr int NOFF = BITS == 2 ? 5 : (BITS == 3 ? 4 : (BITS == 4 ? 2 : 1));  // distinct offsets 0, step, 2*step, ...
-    constexpr int OSTEP = BITS == 4 ? 4 : 2;
+    constexpr int BIAS = BITS == 2 ? 4 : (BITS == 3 ? 3 : ((BITS == 4 || BITS == 6) ? 2 : 0));
+    constexpr int NOFF = BITS == 2 ? 5 : (BITS == 3 ? 4 : ((BITS == 4 || BITS == 6) ? 2 : 1));  // distinct offsets 0, step, 2*step, ...
+    constexpr int OSTEP = (BITS == 4 || BITS == 6) ? 4 : 2;
     const uint32_t* prm = reinterpret_cast<const uint32_t*>(st + 8 * atom_bytes(BITS));
     const __half2 k1024 = __float2half2_rn(1024.f);
     Codes<BITS> cd;
@@ -406,6 +406,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
                         case 2: t2_dequant_half<2>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<2>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
                         case 3: t2_dequant_half<3>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<3>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
                         case 4: t2_dequant_half<4>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<4>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
+                        case 6: t2_dequant_half<6>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<6>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
                         default: t2_dequant_half<8>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<8>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
                     }
                 } else {

@@ -25,6 +25,12 @@
 //          phi <= 1 in place (o = 4phi), phi >= 2 after >> 8 (o = 4phi - 8): o = 4h.
 //   8-bit: atom = 4 planes x [32 lanes x 16 B]; plane s/2, word 2*(s%2) + h; byte 2*rowhalf + odd
 //          (expanded with one byte permute per pair; o = 0).
+//   6-bit: low four bits stored exactly as a 4-bit atom (1024 B, o = 4h), then a 2-bit plane [32 lanes x 16 B] with
+//          the high two bits, word jh*2 + rowhalf as in a 2-bit atom.  The high bits of step s4 = s%4, pair h must
+//          land on bits [o+4, o+6) = 4 + 4h (even k; +16 odd k) of a copy of that word: the copies are the word
+//          itself (s4 = 0), the word >> 2 (s4 = 1), the word with the bytes of each half swapped (s4 = 2) and that
+//          one >> 2 (s4 = 3), so the field is stored at bit (4 + 4h + {0, 2, 8, 10}[s4]) % 16 of its half.  The
+//          eight fields of a half tile its sixteen bits exactly.
 #pragma once
 #include <stdint.h>
 
@@ -36,7 +42,8 @@ struct CodeLoc {
     int width;     // field width
 };
 
-// r: row in atom (0..15), kk: k in chunk (0..127).  For 3-bit, part 0 = low two bits, part 1 = high bit.
+// r: row in atom (0..15), kk: k in chunk (0..127).  For 3-bit, part 0 = low two bits, part 1 = high bit; for
+// 6-bit, part 0 = low four bits, part 1 = high two bits.
 __host__ __device__ inline CodeLoc code_loc(int bits, int r, int kk, int part) {
     const int gid = r & 7, rowhalf = r >> 3;
     const int s = kk >> 4, kq = kk & 15;
@@ -44,7 +51,12 @@ __host__ __device__ inline CodeLoc code_loc(int bits, int r, int kk, int part) {
     const int lane = gid * 4 + tid4;
     const int jh = s >> 2, s4 = s & 3;
     CodeLoc L;
-    if (bits == 4) {
+    if (bits == 6 && part == 1) {  // 6-bit, high two bits
+        const int rot = (s4 & 1) * 2 + (s4 >> 1) * 8;
+        L.byte_off = 1024 + lane * 16 + (jh * 2 + rowhalf) * 4;
+        L.shift = ((4 + 4 * h + rot) & 15) + 16 * odd;
+        L.width = 2;
+    } else if (bits == 4 || bits == 6) {
         const int phi = 2 * (s4 & 1) + h;
         L.byte_off = jh * 512 + lane * 16 + (rowhalf * 2 + (s4 >> 1)) * 4;
         L.shift = 4 * phi + 16 * odd;
@@ -72,14 +84,16 @@ __host__ __device__ inline CodeLoc code_loc(int bits, int r, int kk, int part) {
 
 // Activations feeding a matrix packed at `bits` are stored multiplied by 2^x_scale_exp(bits, k):
 // bias - o(k), with o the in-place bit offset of the code of input index k (periodic in k mod 64).
-__host__ __device__ inline int x_scale_bias(int bits) { return bits == 2 ? 4 : (bits == 3 ? 3 : (bits == 4 ? 2 : 0)); }
+__host__ __device__ inline int x_scale_bias(int bits) {
+    return bits == 2 ? 4 : (bits == 3 ? 3 : ((bits == 4 || bits == 6) ? 2 : 0));
+}
 __host__ __device__ inline int x_scale_exp(int bits, int k) {
     const int s4 = (k >> 4) & 3, h = (k >> 1) & 1;
     const int phi = 2 * s4 + h;
     int o = 0;
     if (bits == 2) o = phi <= 4 ? 2 * phi : 2 * phi - 10;
     else if (bits == 3) o = 2 * (phi & 3);
-    else if (bits == 4) o = 4 * h;
+    else if (bits == 4 || bits == 6) o = 4 * h;
     return x_scale_bias(bits) - o;
 }
 

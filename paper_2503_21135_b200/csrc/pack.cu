@@ -51,10 +51,11 @@ __global__ void __launch_bounds__(256) pack_blocks_kernel(const __nv_bfloat16* _
         for (int i = 0; i < G; ++i) {
             const int kk = g * G + i;
             const int q = quantize_code(bf16_to_double(p[kk]), s, m, bits);
-            if (bits == 3) {
-                CodeLoc a = code_loc(3, ra, kk, 0), b = code_loc(3, ra, kk, 1);
-                atomicOr(&atom_words[a.byte_off >> 2], (uint32_t)(q & 3) << a.shift);
-                atomicOr(&atom_words[b.byte_off >> 2], (uint32_t)(q >> 2) << b.shift);
+            if (bits == 3 || bits == 6) {   // two bit planes: the low 2 (4) bits and the high 1 (2) bits
+                const int lowb = bits == 3 ? 2 : 4;
+                CodeLoc a = code_loc(bits, ra, kk, 0), b = code_loc(bits, ra, kk, 1);
+                atomicOr(&atom_words[a.byte_off >> 2], (uint32_t)(q & ((1 << lowb) - 1)) << a.shift);
+                atomicOr(&atom_words[b.byte_off >> 2], (uint32_t)(q >> lowb) << b.shift);
             } else {
                 CodeLoc a = code_loc(bits, ra, kk, 0);
                 atomicOr(&atom_words[a.byte_off >> 2], (uint32_t)q << a.shift);
@@ -181,11 +182,12 @@ __global__ void export_kernel(const LayerDev* __restrict__ L, int e, int mat, in
         const uint8_t* blk = base + ((long long)rb * n_kc + kc) * ex.blk_bytes;
         const uint8_t* atom = blk + (r >> 4) * atom_bytes(bits);
         int code;
-        if (bits == 3) {
-            CodeLoc a = code_loc(3, r & 15, kk, 0), b = code_loc(3, r & 15, kk, 1);
+        if (bits == 3 || bits == 6) {
+            const int lowb = bits == 3 ? 2 : 4;
+            CodeLoc a = code_loc(bits, r & 15, kk, 0), b = code_loc(bits, r & 15, kk, 1);
             const uint32_t wa = *reinterpret_cast<const uint32_t*>(atom + a.byte_off);
             const uint32_t wb = *reinterpret_cast<const uint32_t*>(atom + b.byte_off);
-            code = ((wa >> a.shift) & 3) | (((wb >> b.shift) & 1) << 2);
+            code = ((wa >> a.shift) & ((1u << lowb) - 1)) | (((wb >> b.shift) & ((1u << (bits - lowb)) - 1)) << lowb);
         } else {
             CodeLoc a = code_loc(bits, r & 15, kk, 0);
             const uint32_t wa = *reinterpret_cast<const uint32_t*>(atom + a.byte_off);

@@ -104,8 +104,10 @@ def test_pack_argument_errors_detected_before_any_launch(lib):
         h, k.get("wg", args["w"]), args["w"], args["w"], k.get("bits", bits), k.get("pool", pool),
         k.get("arena", args["arena"]), k.get("nbytes", args["nbytes"]), args["arena"], args["nbytes"], None)
     assert call(wg=None) == 1
-    bad = bits.copy(); bad[3] = 6
+    bad = bits.copy(); bad[3] = 5
     assert call(bits=bad) == 3
+    six = bits.copy(); six[3] = 6                      # INT6 is a base width
+    assert binding.dynamo_arena_bytes(_desc(), six)[0] == 0
     p2 = pool.copy(); p2[2, 5] = p2[2, 4]
     assert call(pool=p2) == 7
     p3 = pool.copy(); p3[1, 63] = 512

@@ -1,6 +1,6 @@
 """GPU parity on odd layer shapes and degenerate settings, every token against the oracle: dimensions that are the
 smallest multiples the layout allows, top-k at its maximum, a cache pool that is not a multiple of 32, no channel
-cache at all, only 8-bit experts, a shared expert, empty experts, token counts of 0 and 1."""
+cache at all, only 8-bit experts, 6-bit experts, a shared expert, empty experts, token counts of 0 and 1."""
 import numpy as np
 import pytest
 import torch
@@ -24,6 +24,13 @@ CASES = {
                               cache_size=0, bits=[2, 3, 4, 2], tokens=(5, 90)),
     "topk8_pool_not_multiple_of_32": dict(d_model=1024, d_ff=640, n_experts=16, top_k=8, group_size=64, n_shared=0,
                                           max_sig=48, cache_size=48, bits=[2, 3, 4, 8] * 4, tokens=(3, 130)),
+    # INT6 as the base width of whole experts (Section IV-A: INT2/4/6/8), at both group sizes, with and without cache
+    "int6_base_g128": dict(d_model=1024, d_ff=512, n_experts=8, top_k=2, group_size=128, n_shared=0, max_sig=32,
+                           cache_size=64, bits=[2, 3, 4, 6, 6, 4, 8, 6], tokens=(1, 7, 40, 200)),
+    "int6_base_g64_shared": dict(d_model=768, d_ff=384, n_experts=4, top_k=2, group_size=64, n_shared=1, max_sig=16,
+                                 cache_size=32, bits=[6, 6, 6, 2], tokens=(3, 150)),
+    "int6_only_no_cache": dict(d_model=256, d_ff=128, n_experts=2, top_k=1, group_size=128, n_shared=0, max_sig=0,
+                               cache_size=0, bits=[6, 6], tokens=(1, 90)),
     "one_expert": dict(d_model=512, d_ff=256, n_experts=1, top_k=1, group_size=128, n_shared=0, max_sig=8, cache_size=40,
                        bits=[3], tokens=(2, 100)),
 }
@@ -43,12 +50,13 @@ def test_shape(name):
     sets = wl.initial_sig_sets(cfg, pool)
     gpu.set_channel_switch(sets)
     ora.set_channel_switch(sets)
-    # codes of every expert's gate matrix, bit for bit
+    # codes of every expert's gate matrix, and of all three matrices of the 6-bit experts, bit for bit
     for e in range(cfg.n_experts + cfg.n_shared):
-        q, s, m = gpu.export_codes(e, binding.MAT_GATE)
-        assert torch.equal(q.cpu(), torch.from_numpy(ora.base[e][0].q)), e
-        assert np.array_equal(s.cpu().numpy().view(np.uint16), ora.base[e][0].s)
-        assert np.array_equal(m.cpu().numpy().view(np.uint16), ora.base[e][0].m)
+        for mat in ((binding.MAT_GATE, binding.MAT_UP, binding.MAT_DOWN) if bits[e] == 6 else (binding.MAT_GATE,)):
+            q, s, m = gpu.export_codes(e, mat)
+            assert torch.equal(q.cpu(), torch.from_numpy(ora.base[e][mat].q)), (e, mat)
+            assert np.array_equal(s.cpu().numpy().view(np.uint16), ora.base[e][mat].s)
+            assert np.array_equal(m.cpu().numpy().view(np.uint16), ora.base[e][mat].m)
     for step, T in enumerate(tokens):
         x, lg = wl.activations(cfg, T, step=step), wl.router_logits(cfg, T, step=step)
         y, dbg = gpu.forward(x.cuda(), lg.cuda(), binding.F32, debug=True)

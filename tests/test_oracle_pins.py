@@ -145,7 +145,7 @@ def test_dequantize_matches_numpy_formula():
 
 # ---- C2 packing --------------------------------------------------------------------------
 
-@pytest.mark.parametrize("bits", [2, 3, 4, 8])
+@pytest.mark.parametrize("bits", [2, 3, 4, 6, 8])
 @pytest.mark.parametrize("K", [32, 33, 64, 100, 128, 384])
 def test_pack_roundtrip(bits, K):
     rng = np.random.default_rng(bits * 1000 + K)
@@ -175,7 +175,7 @@ def test_pack_bit_positions_hand_example():
 
 
 def test_groups_stay_word_aligned():
-    for G, bits in itertools.product((64, 128), (2, 3, 4, 8)):
+    for G, bits in itertools.product((64, 128), (2, 3, 4, 6, 8)):
         assert (G * bits) % 32 == 0
 
 
