@@ -211,6 +211,16 @@ dynamo_status dynamo_poll_status(dynamo_ctx* ctx, void* stream);
 dynamo_status dynamo_debug_expire_wait(dynamo_ctx* ctx, int64_t limit_ns, void* stream);
 dynamo_status dynamo_debug_check_guards(dynamo_ctx* ctx, int64_t* n_bad_bytes, void* stream);
 
+/* Operand precision of the tensor-core products (Section V-B dequantizes to FP16; a bf16 pipeline is the other
+ * common choice).  Integer codes up to 255 and bf16 inputs are exact in fp16 and in bf16, and every product is exact
+ * in the fp32 accumulator, so the two formats differ in ONE place: the hidden activations h = silu(g) * u, which
+ * are the second projection's operand.  DYNAMO_OPERAND_FP16 (default) rounds h to fp16 (11 significant bits),
+ * DYNAMO_OPERAND_BF16 rounds it to bf16 (8 significant bits; every bf16 value inside the operand range is an fp16
+ * value, so the same instruction then computes what bf16 operands give).  Host-side setting, takes effect with the
+ * next forward; costs one conversion per hidden value.  Errors: NULL ctx -> ERR_NULL; another value -> ERR_ARG. */
+enum { DYNAMO_OPERAND_FP16 = 0, DYNAMO_OPERAND_BF16 = 1 };
+dynamo_status dynamo_set_operand_dtype(dynamo_ctx* ctx, int32_t operand_dtype);
+
 /* Path selection: experts that receive more than `rows` tokens in a forward run on the tcgen05
  * (tensor-memory) kernel, the others on the streaming kernel.  Default 32 (also the maximum);
  * 0 switches the tcgen05 path off.  Both paths implement the same arithmetic definition. */

@@ -240,6 +240,16 @@ class OracleLayer:
             if self.base[e] is not None and self.bits[e] < HI_BITS:
                 self.hi_down[e] = QuantMatrix(*quantize(w_down[e], self.G, HI_BITS))
 
+    def set_channel_precision_down(self, hi_bits: Sequence[int], w_down) -> None:
+        """Precision the significant hidden units are served at, per routed expert (Section IV-B, as
+        ``set_channel_precision`` but for the input channels of W_down): a significant hidden unit of expert e
+        takes the column it has in the expert's uniform hi_bits[e]-bit quantization of the ORIGINAL W_down
+        (same groups, same quantizer).  w_down: the original bf16 bit patterns [E+Es, d, f]."""
+        assert len(hi_bits) == self.E
+        for e in range(self.E):
+            if self.hi_down[e] is not None:
+                self.hi_down[e] = QuantMatrix(*quantize(w_down[e], self.G, int(hi_bits[e])))
+
     def set_channel_switch_down(self, sets: Sequence[np.ndarray]) -> None:
         """Install the significant set of W_down's input channels (indices in [0, f)) of every routed expert."""
         assert len(sets) == self.E

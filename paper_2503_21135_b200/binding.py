@@ -22,6 +22,7 @@ _lib = None
 OK = 0
 BF16, F32 = 0, 1
 MAT_GATE, MAT_UP, MAT_DOWN = 0, 1, 2
+OPERAND_FP16, OPERAND_BF16 = 0, 1
 CODES_BASE, CODES_HI_POOL, CODES_HI_ACTIVE = 0, 1, 2
 SWITCH_SELECT, SWITCH_REQUANT = 0, 1
 
@@ -31,7 +32,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_BITS", "ERR_ALIGN", "ERR_ARE
 EXPORTED = ["dynamo_create", "dynamo_destroy", "dynamo_arena_bytes", "dynamo_pack_experts",
             "dynamo_set_channel_switch", "dynamo_set_channel_switch_many", "dynamo_set_switch_mode",
             "dynamo_moe_forward", "dynamo_moe_forward_router", "dynamo_moe_forward_host", "dynamo_export_codes", "dynamo_expert_stream_bytes",
-            "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_stats_collection", "dynamo_set_channel_precision", "dynamo_assign_bits",
+            "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_operand_dtype", "dynamo_set_stats_collection", "dynamo_set_channel_precision", "dynamo_assign_bits",
             "dynamo_down_cache_bytes", "dynamo_pack_down_cache", "dynamo_set_channel_switch_down",
             "dynamo_get_channel_stats", "dynamo_select_significant", "dynamo_route_permute_static",
             "dynamo_debug_expire_wait", "dynamo_debug_check_guards",
@@ -80,6 +81,7 @@ def load():
         L.dynamo_poll_status.argtypes = [vp, vp]
         L.dynamo_set_profile_events.argtypes = [vp, vp, vp, vp]
         L.dynamo_set_tc_min_rows.argtypes = [vp, i32]
+        L.dynamo_set_operand_dtype.argtypes = [vp, i32]
         L.dynamo_set_stats_collection.argtypes = [vp, i32]
         L.dynamo_set_channel_precision.argtypes = [vp, i32p, vp]
         L.dynamo_down_cache_bytes.argtypes = [vp, i32p, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
@@ -180,6 +182,10 @@ def dynamo_poll_status(ctx, stream) -> int:
 
 def dynamo_set_tc_min_rows(ctx, rows: int) -> int:
     return load().dynamo_set_tc_min_rows(ctx, rows)
+
+
+def dynamo_set_operand_dtype(ctx, operand_dtype: int) -> int:
+    return load().dynamo_set_operand_dtype(ctx, operand_dtype)
 
 
 def dynamo_set_profile_events(ctx, e0, e1, e2) -> int:
@@ -373,6 +379,10 @@ class DynamoLayer:
 
     def set_tc_min_rows(self, rows: int):
         _check(dynamo_set_tc_min_rows(self.ctx, rows), "dynamo_set_tc_min_rows")
+
+    def set_operand_dtype(self, operand_dtype: int):
+        """OPERAND_FP16 (default) or OPERAND_BF16: precision the hidden activations carry into the second projection."""
+        _check(dynamo_set_operand_dtype(self.ctx, operand_dtype), "dynamo_set_operand_dtype")
 
     def set_channel_precision(self, hi_bits):
         """Precision the significant channels of each routed expert are served at: int [E], each in {2,3,4,6,8}."""

@@ -247,6 +247,7 @@ struct dynamo_ctx {
     LayerDev host_layer;                         // host mirror of the arena header
     int switch_mode = DYNAMO_SWITCH_SELECT;
     int tc_min_rows = TC_MIN_ROWS;               // experts with more rows take the tcgen05 path
+    int operand_dtype = DYNAMO_OPERAND_FP16;     // precision the hidden activations carry into the down GEMM
     int collect_stats = 0;                       // 1: every forward adds to the per-channel activation statistics
     int n_sms = 148;                             // SM count of the device the layer was packed on
     int tc2_clusters[2] = {0, 0};                // resident CTA pairs of the tcgen05 kernel there (down, gate/up)
@@ -283,6 +284,7 @@ WsDev make_ws(const dynamo_ctx* c, int T) {
     // No expert can exceed T rows.  Up to twice the threshold the streaming kernel takes a large expert as
     // chunks of 24 tokens (the later passes over its blocks hit L2), which costs less than two more launches.
     w.tc_min = (c->tc_min_rows != 0x7fffffff && T > 2 * c->tc_min_rows) ? c->tc_min_rows : 0x7fffffff;
+    w.h_bf16 = c->operand_dtype == DYNAMO_OPERAND_BF16;
     return w;
 }
 
@@ -383,6 +385,13 @@ dynamo_status dynamo_set_profile_events(dynamo_ctx* ctx, void* before_gateup, vo
     ctx->prof_ev[0] = (cudaEvent_t)before_gateup;
     ctx->prof_ev[1] = (cudaEvent_t)after_gateup;
     ctx->prof_ev[2] = (cudaEvent_t)after_down;
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_set_operand_dtype(dynamo_ctx* ctx, int32_t operand_dtype) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    if (operand_dtype != DYNAMO_OPERAND_FP16 && operand_dtype != DYNAMO_OPERAND_BF16) return DYNAMO_ERR_ARG;
+    ctx->operand_dtype = operand_dtype;
     return DYNAMO_OK;
 }
 

@@ -90,6 +90,7 @@ struct WsDev {
     int32_t Rpad;
     int32_t Rcap;         // rows allocated in the activation buffers (their chunk pitch)
     int32_t tc_min;       // experts with more rows than this take the tcgen05 path (INT_MAX: none)
+    int32_t h_bf16;       // 1: hidden activations are rounded to bf16 before they become the down GEMM's operand
 };
 
 // Activation layouts.  Both give a row group of 8 rows the same footprint (8 * XROW bytes per 128-k
@@ -136,6 +137,14 @@ __device__ __forceinline__ float clamp_act(float v, bool& hit) {
         v = copysignf(ACT_LIMIT, v);
     }
     return v;
+}
+
+// Operand precision of the hidden activations.  The integer codes (at most 255) and the bf16 inputs are exact in
+// fp16 and in bf16 alike and every product is exact in the fp32 accumulator, so the hidden value h is the one
+// operand on which a bf16 tensor-core path and an fp16 one differ: rounding h to bf16 (an exact fp16 value inside
+// the clamp range) gives the arithmetic of bf16 operands on the fp16 instruction.
+__device__ __forceinline__ float round_operand(float h, int to_bf16) {
+    return to_bf16 ? __bfloat162float(__float2bfloat16_rn(h)) : h;
 }
 
 // ---- PTX helpers -----------------------------------------------------------------------

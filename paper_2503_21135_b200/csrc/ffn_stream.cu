@@ -253,6 +253,7 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
                     float h = g / (1.f + expf(-g)) * u;
                     const int tok = 8 * j + 2 * tid4 + c;
                     if (tok < im.nvalid) h = clamp_act(h, clamped);   // columns past the last token hold stale data
+                    h = round_operand(h, p.ws.h_bf16);
                     *reinterpret_cast<__half*>(htile + tok * XROW + (8 * (atom0 + a) + gid) * 2) = __float2half_rn(h);
                 }
         __syncwarp();

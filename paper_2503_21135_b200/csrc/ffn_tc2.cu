@@ -458,6 +458,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
                                 const float v0 = __uint_as_float(r[4 * j + c]), v1 = __uint_as_float(r[4 * j + 2 + c]);
                                 float h = __fdividef(v0, 1.f + __expf(-v0)) * v1;
                                 if (n0 + c < w.n_valid) h = clamp_act(h, clamped);   // columns past the last token: ignored
+                                h = round_operand(h, p.ws.h_bf16);
                                 hs[c] = __half2float(__float2half_rn(h)) * scl;   // exact: scl is a power of two
                             }
                             const int odd = gid & 1;

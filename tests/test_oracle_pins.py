@@ -395,6 +395,33 @@ def test_down_side_set_brute_force_and_identities():
     assert np.array_equal(layer.forward(x, logits)["y"], base)
 
 
+@pytest.mark.parametrize("hb", [3, 4, 6])
+def test_down_side_precision_all_switched_equals_uniform_target(hb):
+    # every hidden unit significant at target hb: W_down is the expert's uniform hb-bit quantization (gate/up stay
+    # at their base); a target equal to the base bit-width changes nothing; going back to 8 restores the state
+    layer, x, logits, (wg, wu, wd) = _tiny_layer(seed=15, bits=(2, 3, 2, 8))
+    ud = bf16_bits(wd)
+    layer.enable_down_side(ud)
+    some = [np.arange(0, layer.f, 5)] * 4
+    layer.set_channel_switch_down(some)
+    y8 = layer.forward(x, logits)["y"]
+    layer.set_channel_precision_down([hb] * 4, ud)
+    assert layer.hi_down[3] is None                              # the 8-bit expert has no switch
+    ref = oracle.OracleLayer(bf16_bits(wg), bf16_bits(wu), ud, [hb, hb, hb, 8], layer.G, 4, 2)
+    for e in range(3):
+        ref.base[e] = (layer.base[e][0], layer.base[e][1], ref.base[e][2])
+    layer.set_channel_switch_down([np.arange(layer.f)] * 4)
+    assert np.array_equal(layer.forward(x, logits)["y"], ref.forward(x, logits)["y"])
+    if hb == 3:                                                  # expert 1 is 3-bit already: its set has no effect
+        _, _, d0 = layer.effective_weights(1)
+        layer.set_channel_switch_down([np.array([], np.int32)] * 4)
+        _, _, d1 = layer.effective_weights(1)
+        assert np.array_equal(d0, d1)
+    layer.set_channel_precision_down([8] * 4, ud)
+    layer.set_channel_switch_down(some)
+    assert np.array_equal(layer.forward(x, logits)["y"], y8)
+
+
 def test_empty_set_is_base_and_8bit_expert_ignores_mask():
     layer, x, logits, _ = _tiny_layer(seed=6)           # expert 3 is 8-bit
     base = layer.forward(x, logits)["y"]
