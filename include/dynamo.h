@@ -272,16 +272,28 @@ dynamo_status dynamo_select_significant(dynamo_ctx* ctx, int32_t n_select, int32
  * dynamo_pack_down_cache: after dynamo_pack_experts (a new dynamo_pack_experts drops the cache).
  *   w_down         : device bf16 [E + E_s, d_model, d_ff], the originals given to dynamo_pack_experts
  *   cache_idx_down : host int32 [E, cache_size_down], strictly increasing per expert, each in [0, d_ff)
- *   Builds the 8-bit parameters of every (row, group) of W_down and, per cached hidden unit, its 8-bit codes, bf16
- *   originals (the channel cache) and differences.  All sets start empty.  Synchronises the stream.
+ *   Builds the 8-bit parameters and the extrema of every (row, group) of W_down and, per cached hidden unit, its
+ *   8-bit codes, bf16 originals (the channel cache) and differences.  All sets start empty.  Synchronises the stream.
  * dynamo_set_channel_switch_down: installs the sets (the state depends only on the last call).
  *   sig_idx : host int32 [E, max_sig_down], sig_cnt : host int32 [E], 0 <= cnt <= max_sig_down
  *   8-bit experts are validated but keep the empty set.  Stream-ordered like dynamo_set_channel_switch: a switch
  *   enqueued between two forwards takes effect exactly between them (the tables travel by three small copies from
  *   pageable host memory, which the CUDA runtime stages before the call returns).
- * dynamo_export_codes with DYNAMO_MAT_DOWN and DYNAMO_CODES_HI_POOL / HI_ACTIVE returns the 8-bit codes of the
- * cached / significant hidden units (0 elsewhere) and the 8-bit parameters, shaped like the base export.
- * dynamo_set_channel_precision does not reach this side: it stays at 8 bits.
+ *   In switch mode DYNAMO_SWITCH_REQUANT one more kernel re-derives codes and differences of the new sets'
+ *   channels from the bf16 channel cache at the expert's target precision (channel replacement followed by
+ *   requantization, Section IV-B); the resulting state equals the one DYNAMO_SWITCH_SELECT reaches, bit for bit.
+ * dynamo_set_channel_precision_down: precision the significant hidden units are served at (Section IV-B: requantized
+ *   to the precision the new data calls for, higher or lower than before); the d_ff-side twin of
+ *   dynamo_set_channel_precision, which does not reach this side.
+ *   hi_bits : host int32 [E], each in {2, 3, 4, 6, 8}; 8 for every expert after dynamo_pack_down_cache.
+ *   For every routed expert with base bits < 8 whose value changes, one kernel recomputes from the stored group
+ *   extrema the parameters of the expert's uniform hi_bits[e]-bit quantization of W_down and, from the bf16 channel
+ *   cache, the code and the difference to the base value of every cached hidden unit.  A target equal to the base
+ *   bit-width makes every difference zero; going back to 8 restores the packed state bit for bit.  Stream-ordered.
+ *   Errors: a value outside {2, 3, 4, 6, 8} -> ERR_BITS (nothing changes).
+ * dynamo_export_codes with DYNAMO_MAT_DOWN and DYNAMO_CODES_HI_POOL / HI_ACTIVE returns the codes of the cached /
+ * significant hidden units at the current target precision (0 elsewhere) and that precision's parameters, shaped
+ * like the base export.
  * Errors: NULL -> ERR_NULL; before dynamo_pack_experts (or, for the switch and the export, before
  * dynamo_pack_down_cache) -> ERR_STATE; cache_size_down outside [1, min(d_ff, 65535)], max_sig_down outside
  * [0, min(256, cache_size_down)] -> ERR_SHAPE; arena misaligned -> ERR_ALIGN, too small -> ERR_ARENA_TOO_SMALL; an
@@ -292,6 +304,7 @@ dynamo_status dynamo_down_cache_bytes(const dynamo_layer_desc* desc, const int32
 dynamo_status dynamo_pack_down_cache(dynamo_ctx* ctx, const void* w_down, const int32_t* cache_idx_down,
                                      int32_t cache_size_down, int32_t max_sig_down, void* down_arena, size_t down_bytes,
                                      void* stream);
+dynamo_status dynamo_set_channel_precision_down(dynamo_ctx* ctx, const int32_t* hi_bits, void* stream);
 dynamo_status dynamo_set_channel_switch_down(dynamo_ctx* ctx, const int32_t* sig_idx, const int32_t* sig_cnt,
                                              void* stream);
 

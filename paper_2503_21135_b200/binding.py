@@ -34,6 +34,7 @@ EXPORTED = ["dynamo_create", "dynamo_destroy", "dynamo_arena_bytes", "dynamo_pac
             "dynamo_moe_forward", "dynamo_moe_forward_router", "dynamo_moe_forward_host", "dynamo_export_codes", "dynamo_expert_stream_bytes",
             "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_operand_dtype", "dynamo_set_stats_collection", "dynamo_set_channel_precision", "dynamo_assign_bits",
             "dynamo_down_cache_bytes", "dynamo_pack_down_cache", "dynamo_set_channel_switch_down",
+            "dynamo_set_channel_precision_down",
             "dynamo_get_channel_stats", "dynamo_select_significant", "dynamo_route_permute_static",
             "dynamo_debug_expire_wait", "dynamo_debug_check_guards",
             "dynamo_kernel_launches", "dynamo_status_str"]
@@ -84,6 +85,7 @@ def load():
         L.dynamo_set_operand_dtype.argtypes = [vp, i32]
         L.dynamo_set_stats_collection.argtypes = [vp, i32]
         L.dynamo_set_channel_precision.argtypes = [vp, i32p, vp]
+        L.dynamo_set_channel_precision_down.argtypes = [vp, i32p, vp]
         L.dynamo_down_cache_bytes.argtypes = [vp, i32p, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
         L.dynamo_pack_down_cache.argtypes = [vp, vp, i32p, i32, i32, vp, ctypes.c_size_t, vp]
         L.dynamo_set_channel_switch_down.argtypes = [vp, i32p, i32p, vp]
@@ -389,6 +391,13 @@ class DynamoLayer:
         hb = np.ascontiguousarray(np.asarray(hi_bits, dtype=np.int32))
         assert hb.shape == (self.desc.n_experts,)
         _check(load().dynamo_set_channel_precision(self.ctx, _i32p(hb), _stream()), "dynamo_set_channel_precision")
+
+    def set_channel_precision_down(self, hi_bits):
+        """Precision the significant hidden units (d_ff side) of each routed expert are served at: int [E]."""
+        hb = np.ascontiguousarray(np.asarray(hi_bits, dtype=np.int32))
+        assert hb.shape == (self.desc.n_experts,)
+        _check(load().dynamo_set_channel_precision_down(self.ctx, _i32p(hb), _stream()),
+               "dynamo_set_channel_precision_down")
 
     def set_stats_collection(self, on: bool):
         _check(load().dynamo_set_stats_collection(self.ctx, int(bool(on))), "dynamo_set_stats_collection")

@@ -17,6 +17,10 @@ cudaError_t launch_retarget(LayerDev* L, int e, int f, int bits, cudaStream_t st
 cudaError_t launch_pack_down_hi(const void* w_down, int d, int f, int G, int P2, const int32_t* cache_idx_dev,
                                 int base_bits, const DownExpertDev& ex, cudaStream_t st);
 cudaError_t launch_down_fix(const LayerDev* L, const DownDev* D2, const WsDev& ws, int d, cudaStream_t st);
+cudaError_t launch_retarget_down(int d, int f, int G, int P2, const int32_t* cache_idx_dev, int base_bits, int hi_bits,
+                                 const DownExpertDev& ex, cudaStream_t st);
+cudaError_t launch_requant_down(const LayerDev* L, const DownDev* D2, const int32_t* hi_bits_dev, int d, int n_experts,
+                                cudaStream_t st);
 cudaError_t launch_export_down(const LayerDev* L, const DownDev* D2, int e, int which, long long n_elems, uint8_t* q,
                                uint16_t* sc, uint16_t* zr, cudaStream_t st);
 cudaError_t launch_export(const LayerDev* L, int e, int mat, int which, long long n_elems, uint8_t* q, uint16_t* sc,
@@ -86,8 +90,8 @@ inline int switch_ints_per_layer(const dynamo_layer_desc& D) { return D.n_expert
 // Arena of the d_ff-side channel cache: header, tables, then per switchable expert the 8-bit parameters of W_down,
 // the cached channels' codes, differences and bf16 originals.
 struct DownLayout {
-    size_t cache_idx = 0, sig_chan = 0, sig_pool = 0, sig_cnt = 0;
-    std::vector<size_t> s8m8, q8, delta, cache_w;
+    size_t cache_idx = 0, sig_chan = 0, sig_pool = 0, sig_cnt = 0, hi_bits = 0;
+    std::vector<size_t> s8m8, gminmax, q8, delta, cache_w;
     size_t total = 0;
 };
 
@@ -99,10 +103,12 @@ void down_layout(const dynamo_layer_desc& D, const int32_t* bits, int P2, int S2
     A.sig_chan = take(E * (size_t)std::max(S2, 1) * 4);
     A.sig_pool = take(E * (size_t)std::max(S2, 1) * 4);
     A.sig_cnt = take(E * 4);
-    A.s8m8.assign(E, 0); A.q8.assign(E, 0); A.delta.assign(E, 0); A.cache_w.assign(E, 0);
+    A.hi_bits = take(E * 4);
+    A.s8m8.assign(E, 0); A.gminmax.assign(E, 0); A.q8.assign(E, 0); A.delta.assign(E, 0); A.cache_w.assign(E, 0);
     for (size_t e = 0; e < E; ++e) {
         if (bits[e] >= HI_BITS) continue;
         A.s8m8[e] = take(d * (f / G) * 4);
+        A.gminmax[e] = take(d * (f / G) * 4);
         A.q8[e] = take((size_t)P2 * d);
         A.delta[e] = take((size_t)P2 * d * 2);
         A.cache_w[e] = take((size_t)P2 * d * 2);
@@ -237,6 +243,8 @@ struct dynamo_ctx {
     DownLayout DA;
     std::vector<int32_t> cache_idx_down;         // host copy [E][P2]
     std::vector<std::vector<int32_t>> sig_down;  // current sets, in slot order
+    std::vector<int32_t> hi_bits_down;           // precision the significant hidden units of each routed expert are served at
+    std::vector<uint8_t> down_hdr;               // host copy of the d_ff-side cache's device header
     int down_active = 0;                         // experts whose d_ff-side set is not empty
     std::vector<int32_t> cache_idx;              // host copy [E][P]
     std::vector<std::vector<int32_t>> sig;       // current sets, in slot order
@@ -803,6 +811,7 @@ dynamo_status dynamo_pack_down_cache(dynamo_ctx* ctx, const void* w_down, const 
     ctx->DA = A;
     ctx->cache_idx_down.assign(cache_idx_down, cache_idx_down + (size_t)E * P2);
     ctx->sig_down.assign(E, {});
+    ctx->hi_bits_down.assign(E, HI_BITS);
 
     std::vector<uint8_t> hdr(sizeof(DownDev), 0);
     DownDev& H = *reinterpret_cast<DownDev*>(hdr.data());
@@ -815,6 +824,7 @@ dynamo_status dynamo_pack_down_cache(dynamo_ctx* ctx, const void* w_down, const 
     for (int e = 0; e < E; ++e) {
         if (ctx->bits[e] >= HI_BITS) continue;
         H.ex[e].s8m8 = (uint32_t*)(base + A.s8m8[e]);
+        H.ex[e].gminmax = (uint32_t*)(base + A.gminmax[e]);
         H.ex[e].q8 = base + A.q8[e];
         H.ex[e].delta = (__half*)(base + A.delta[e]);
         H.ex[e].cache_w = (__nv_bfloat16*)(base + A.cache_w[e]);
@@ -824,6 +834,7 @@ dynamo_status dynamo_pack_down_cache(dynamo_ctx* ctx, const void* w_down, const 
     CUDA_TRY(cudaMemsetAsync(H.sig_chan, 0xff, (size_t)E * H.S2 * 4, st));
     CUDA_TRY(cudaMemsetAsync(H.sig_pool, 0, (size_t)E * H.S2 * 4, st));
     CUDA_TRY(cudaMemsetAsync(H.sig_cnt, 0, (size_t)E * 4, st));
+    CUDA_TRY(cudaMemcpyAsync(base + A.hi_bits, ctx->hi_bits_down.data(), (size_t)E * 4, cudaMemcpyHostToDevice, st));
     const char* wd = (const char*)w_down;
     const size_t per_expert = (size_t)D.d_model * D.d_ff * 2;
     for (int e = 0; e < E; ++e) {
@@ -834,6 +845,32 @@ dynamo_status dynamo_pack_down_cache(dynamo_ctx* ctx, const void* w_down, const 
     }
     CUDA_TRY(cudaStreamSynchronize(st));  // the host staging above may go away
     ctx->down_arena = base;
+    ctx->down_hdr = hdr;
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_set_channel_precision_down(dynamo_ctx* ctx, const int32_t* hi_bits, void* stream) {
+    if (!ctx || !hi_bits) return DYNAMO_ERR_NULL;
+    if (!ctx->packed || !ctx->down_arena) return DYNAMO_ERR_STATE;
+    const dynamo_layer_desc& D = ctx->D;
+    for (int e = 0; e < D.n_experts; ++e) {
+        const int b = hi_bits[e];
+        if (b != 2 && b != 3 && b != 4 && b != 6 && b != 8) return DYNAMO_ERR_BITS;  // nothing changes on an error
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    const DownDev& H = *reinterpret_cast<const DownDev*>(ctx->down_hdr.data());
+    bool changed = false;
+    for (int e = 0; e < D.n_experts; ++e) {
+        if (ctx->bits[e] >= HI_BITS || ctx->hi_bits_down[e] == hi_bits[e]) continue;  // 8-bit experts have no cache
+        CUDA_TRY(launch_retarget_down(D.d_model, D.d_ff, D.group_size, ctx->P2, H.cache_idx + (size_t)e * ctx->P2,
+                                      ctx->bits[e], hi_bits[e], H.ex[e], st));
+        ctx->hi_bits_down[e] = hi_bits[e];
+        ctx->launches += 1;
+        changed = true;
+    }
+    if (changed)  // (a copy from pageable memory returns once the source has been staged)
+        CUDA_TRY(cudaMemcpyAsync(ctx->down_arena + ctx->DA.hi_bits, ctx->hi_bits_down.data(), (size_t)D.n_experts * 4,
+                                 cudaMemcpyHostToDevice, st));
     return DYNAMO_OK;
 }
 
@@ -875,6 +912,12 @@ dynamo_status dynamo_set_channel_switch_down(dynamo_ctx* ctx, const int32_t* sig
     ctx->sig_down = lists;
     ctx->down_active = 0;
     for (int e = 0; e < E; ++e) ctx->down_active += cnts[e] > 0 ? 1 : 0;
+    if (ctx->switch_mode == DYNAMO_SWITCH_REQUANT && ctx->down_active > 0) {
+        // channel replacement + requantization: codes and differences of the new sets from the bf16 channel cache
+        CUDA_TRY(launch_requant_down((const LayerDev*)ctx->arena, (const DownDev*)base,
+                                     (const int32_t*)(base + ctx->DA.hi_bits), D.d_model, E, st));
+        ctx->launches += 1;
+    }
     return DYNAMO_OK;
 }
 

@@ -53,9 +53,10 @@ struct LayerDev {
 // Significant set on the d_ff side (Section IV-B applied to the input channels of W_down, the hidden units), kept
 // in its own caller-owned arena so that layers that do not use it pay nothing.
 struct DownExpertDev {
-    uint32_t* s8m8;          // [d][f/G] half2 {scale, zero} of the 8-bit quantization of W_down
-    uint8_t* q8;             // [P2][d] 8-bit codes of the cached channels
-    __half* delta;           // [P2][d] fp16(8-bit value - base value): what a significant channel adds to the base GEMM
+    uint32_t* s8m8;          // [d][f/G] half2 {scale, zero} of W_down's quantization at the target precision (8 after pack)
+    uint32_t* gminmax;       // [d][f/G] two bf16 {min, max} of every group: what another target precision is derived from
+    uint8_t* q8;             // [P2][d] codes of the cached channels at the target precision
+    __half* delta;           // [P2][d] fp16(target value - base value): what a significant channel adds to the base GEMM
     __nv_bfloat16* cache_w;  // [P2][d] bf16 originals of the cached channels (the channel cache)
 };
 struct DownDev {

@@ -7,8 +7,11 @@
 // time as fp16 per (cached channel, output row), so a forward with S2 significant channels per expert costs one
 // small kernel of rows x d x S2 multiply-adds between the down GEMM and the combine, and a switch is a table write.
 //
-// pack   : 8-bit parameters of every (row, group) of W_down; for every cached channel its 8-bit code, its bf16
-//          original (the channel cache) and the fp16 difference to the base value.
+// pack   : 8-bit parameters and the extrema of every (row, group) of W_down; for every cached channel its 8-bit code,
+//          its bf16 original (the channel cache) and the fp16 difference to the base value.
+// retarget: another target precision for an expert's cached channels (Section IV-B: requantized to the precision
+//          the new data calls for): parameters from the stored extrema, codes and differences from the channel cache.
+// requant: the same for the channels of a newly installed set only (switch mode "requantize from the cache").
 // fix    : the correction above, reading h from the activation buffer in the layout the expert's path wrote it in.
 // export : logical 8-bit codes and parameters for parity checks.
 #include "common.cuh"
@@ -37,6 +40,8 @@ __global__ void pack_down_hi_kernel(const __nv_bfloat16* __restrict__ w_down, in
         group_params(lo, hi, HI_BITS, s_h, m_h, s8, m8);
         __half2 pr = __halves2half2(s_h, m_h);
         ex.s8m8[(long long)n * ng + g] = *reinterpret_cast<uint32_t*>(&pr);
+        ex.gminmax[(long long)n * ng + g] = (uint32_t)__bfloat16_as_ushort(__double2bfloat16(lo)) |
+                                            ((uint32_t)__bfloat16_as_ushort(__double2bfloat16(hi)) << 16);
         if (pi < P2 && cache_idx[pi] < (g + 1) * G) {
             double sb, mb;
             group_params(lo, hi, base_bits, s_h, m_h, sb, mb);
@@ -52,6 +57,62 @@ __global__ void pack_down_hi_kernel(const __nv_bfloat16* __restrict__ w_down, in
                 ++pi;
             }
         }
+    }
+}
+
+// Code and difference of cached channel (pool position pi, hidden unit c) in output row n, from the bf16 original:
+// target parameters (s, m) given, base parameters from the group's extrema.
+__device__ __forceinline__ void down_requant_one(const DownExpertDev& ex, int d, int ng, int G, int n, int pi, int c,
+                                                 double s, double m, int hi_bits, int base_bits) {
+    const uint32_t mm = ex.gminmax[(long long)n * ng + c / G];
+    const double lo = bf16_to_double(__ushort_as_bfloat16((unsigned short)(mm & 0xffff)));
+    const double hi = bf16_to_double(__ushort_as_bfloat16((unsigned short)(mm >> 16)));
+    __half s_h, m_h;
+    double sb, mb;
+    group_params(lo, hi, base_bits, s_h, m_h, sb, mb);
+    const double wd = bf16_to_double(ex.cache_w[(long long)pi * d + n]);
+    const int q = quantize_code(wd, s, m, hi_bits);
+    const int qb = quantize_code(wd, sb, mb, base_bits);
+    ex.q8[(long long)pi * d + n] = (uint8_t)q;
+    ex.delta[(long long)pi * d + n] = __double2half((s * (double)q + m) - (sb * (double)qb + mb));
+}
+
+// Another target precision for the cached channels of one expert: one thread per output row n.
+__global__ void retarget_down_kernel(int d, int f, int G, int P2, const int32_t* __restrict__ cache_idx, int base_bits,
+                                     int hi_bits, DownExpertDev ex) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= d) return;
+    const int ng = f / G;
+    int pi = 0;
+    for (int g = 0; g < ng; ++g) {
+        const uint32_t mm = ex.gminmax[(long long)n * ng + g];
+        const double lo = bf16_to_double(__ushort_as_bfloat16((unsigned short)(mm & 0xffff)));
+        const double hi = bf16_to_double(__ushort_as_bfloat16((unsigned short)(mm >> 16)));
+        __half s_h, m_h;
+        double s, m;
+        group_params(lo, hi, hi_bits, s_h, m_h, s, m);
+        __half2 pr = __halves2half2(s_h, m_h);
+        ex.s8m8[(long long)n * ng + g] = *reinterpret_cast<uint32_t*>(&pr);
+        for (; pi < P2 && cache_idx[pi] < (g + 1) * G; ++pi)
+            down_requant_one(ex, d, ng, G, n, pi, cache_idx[pi], s, m, hi_bits, base_bits);
+    }
+}
+
+// Channel replacement followed by requantization for the set just installed (its tables are already on the device in
+// stream order): grid (rows, experts); codes and differences of the set's channels at the expert's target precision.
+__global__ void requant_down_kernel(const LayerDev* __restrict__ L, const DownDev* __restrict__ D2,
+                                    const int32_t* __restrict__ hi_bits) {
+    const int e = blockIdx.y;
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= L->d || !L->ex[e].switchable) return;
+    const DownExpertDev& ex = D2->ex[e];
+    const int ng = L->f / L->G, S2 = D2->S2, cnt = D2->sig_cnt[e];
+    for (int i = 0; i < cnt; ++i) {
+        const int c = D2->sig_chan[(long long)e * S2 + i], pi = D2->sig_pool[(long long)e * S2 + i];
+        const uint32_t prw = ex.s8m8[(long long)n * ng + c / L->G];
+        const __half2 pr = *reinterpret_cast<const __half2*>(&prw);
+        down_requant_one(ex, L->d, ng, L->G, n, pi, c, (double)__low2float(pr), (double)__high2float(pr), hi_bits[e],
+                         L->ex[e].bits);
     }
 }
 
@@ -196,6 +257,18 @@ cudaError_t launch_pack_down_hi(const void* w_down, int d, int f, int G, int P2,
                                 int base_bits, const DownExpertDev& ex, cudaStream_t st) {
     pack_down_hi_kernel<<<(d + 127) / 128, 128, 0, st>>>((const __nv_bfloat16*)w_down, d, f, G, P2, cache_idx_dev,
                                                          base_bits, ex);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_retarget_down(int d, int f, int G, int P2, const int32_t* cache_idx_dev, int base_bits, int hi_bits,
+                                 const DownExpertDev& ex, cudaStream_t st) {
+    retarget_down_kernel<<<(d + 127) / 128, 128, 0, st>>>(d, f, G, P2, cache_idx_dev, base_bits, hi_bits, ex);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_requant_down(const LayerDev* L, const DownDev* D2, const int32_t* hi_bits_dev, int d, int n_experts,
+                                cudaStream_t st) {
+    requant_down_kernel<<<dim3((unsigned)((d + 127) / 128), (unsigned)n_experts), 128, 0, st>>>(L, D2, hi_bits_dev);
     return cudaGetLastError();
 }
 

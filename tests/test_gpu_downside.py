@@ -1,6 +1,6 @@
 """GPU parity for significant channels on the d_ff side (Section IV-B applied to W_down's input channels): 8-bit codes
 and parameters of the cached hidden units bit-exact against the oracle, forwards on every FFN kernel within the output
-tolerance, state = last set installed, error cases."""
+tolerance, state = last set installed, other target precisions, the requantize-from-cache switch mode, error cases."""
 import numpy as np
 import pytest
 import torch
@@ -99,6 +99,105 @@ def test_all_cached_units_on_both_kernels(lay):
             assert rel_err(y.cpu().numpy(), ref) <= TOL
     finally:
         _install(lay, [np.array([], np.int32)] * CFG.n_experts)
+
+
+@pytest.mark.parametrize("target", [6, 4, 3, 2, "mixed"])
+def test_down_side_target_precision(lay, target):
+    """Section IV-B on the d_ff side: the significant hidden units requantized to another precision, higher or lower."""
+    gpu, ora, pool_d = lay["gpu"], lay["ora"], lay["pool_d"]
+    E = CFG.n_experts
+    hb = [6, 2, 4, 3, 8, 6, 4, 2][:E] if target == "mixed" else [target] * E
+    sets = wl.sig_sets_down(CFG, pool_d, S2, event=3)
+    _install(lay, sets)
+    y8 = {T: _forward(lay, T, step=50 + T)[0] for T in (40, 200)}
+    try:
+        gpu.set_channel_precision_down(hb)
+        ora.set_channel_precision_down(hb, oracle.as_u16(lay["wd"]))
+        for e in range(E):
+            if lay["bits"][e] >= 8:
+                continue
+            ref = ora.hi_down[e]
+            q, s, m = gpu.export_codes(e, binding.MAT_DOWN, binding.CODES_HI_POOL)
+            expect = np.zeros_like(ref.q)
+            expect[:, pool_d[e]] = ref.q[:, pool_d[e]]
+            assert np.array_equal(q.cpu().numpy(), expect), e
+            assert int(expect.max()) <= 2 ** hb[e] - 1
+            assert np.array_equal(_u16(s), ref.s) and np.array_equal(_u16(m), ref.m), e
+        for T in (40, 200):                      # streaming kernel only; tcgen05 kernel for the popular experts
+            y, ref = _forward(lay, T, step=50 + T)
+            assert rel_err(y.cpu().numpy(), ref) <= TOL
+        # a target equal to the base bit-width: every difference is zero, the forward is the base forward bit for bit
+        gpu.set_channel_precision_down([int(b) if b < 8 else 8 for b in lay["bits"][:E]])
+        y_same = _forward_gpu_only(lay, 40, 90)
+        _install(lay, [np.array([], np.int32)] * E)
+        assert torch.equal(_forward_gpu_only(lay, 40, 90), y_same)
+        _install(lay, sets)
+    finally:
+        gpu.set_channel_precision_down([8] * E)
+        ora.set_channel_precision_down([8] * E, oracle.as_u16(lay["wd"]))
+    for T in (40, 200):                          # back at 8: the packed state, bit for bit
+        assert torch.equal(_forward(lay, T, step=50 + T)[0], y8[T])
+    _install(lay, [np.array([], np.int32)] * E)
+
+
+def _forward_gpu_only(lay, T, step):
+    x, lg = wl.activations(CFG, T, step=step), wl.router_logits(CFG, T, step=step)
+    y = lay["gpu"].forward(x.cuda(), lg.cuda(), binding.F32)
+    torch.cuda.synchronize()
+    assert lay["gpu"].poll_status() == 0
+    return y
+
+
+def test_down_side_requant_mode_reaches_the_same_state(lay):
+    """Switch mode "requantize from the cache" on the d_ff side: codes and differences of a new set are re-derived
+    from the bf16 channel cache at the current target precision; the state equals the one SELECT mode reaches."""
+    gpu, ora, pool_d = lay["gpu"], lay["ora"], lay["pool_d"]
+    E = CFG.n_experts
+    hb = [4, 6, 3, 6, 8, 2, 4, 6][:E]
+    sets = [wl.sig_sets_down(CFG, pool_d, S2, event=ev) for ev in (5, 6)]
+    try:
+        gpu.set_channel_precision_down(hb)
+        ora.set_channel_precision_down(hb, oracle.as_u16(lay["wd"]))
+        outs = {}
+        for mode in (binding.SWITCH_SELECT, binding.SWITCH_REQUANT):
+            gpu.set_switch_mode(mode)
+            n0 = gpu.kernel_launches()
+            for st in sets:                       # two events in a row: the state depends on the last one only
+                _install(lay, st)
+            if mode == binding.SWITCH_REQUANT:
+                assert gpu.kernel_launches() - n0 == 2      # one requantization launch per event
+            else:
+                assert gpu.kernel_launches() - n0 == 0      # table writes only
+            codes = [tuple(t.clone() for t in gpu.export_codes(e, binding.MAT_DOWN, binding.CODES_HI_ACTIVE))
+                     for e in range(E) if lay["bits"][e] < 8]
+            y, ref = _forward(lay, 40, step=61)
+            assert rel_err(y.cpu().numpy(), ref) <= TOL
+            outs[mode] = (codes, y)
+        for (qa, sa, ma), (qb, sb, mb) in zip(outs[binding.SWITCH_SELECT][0], outs[binding.SWITCH_REQUANT][0]):
+            assert torch.equal(qa, qb) and torch.equal(sa, sb) and torch.equal(ma, mb)
+        assert torch.equal(outs[binding.SWITCH_SELECT][1], outs[binding.SWITCH_REQUANT][1])
+        e0 = next(e for e in range(E) if lay["bits"][e] < 8)
+        q, _, _ = gpu.export_codes(e0, binding.MAT_DOWN, binding.CODES_HI_ACTIVE)
+        expect = np.zeros_like(ora.hi_down[e0].q)
+        expect[:, sets[1][e0]] = ora.hi_down[e0].q[:, sets[1][e0]]
+        assert np.array_equal(q.cpu().numpy(), expect)
+    finally:
+        gpu.set_switch_mode(binding.SWITCH_SELECT)
+        gpu.set_channel_precision_down([8] * E)
+        ora.set_channel_precision_down([8] * E, oracle.as_u16(lay["wd"]))
+        _install(lay, [np.array([], np.int32)] * E)
+
+
+def test_down_side_precision_errors(lay):
+    gpu = lay["gpu"]
+    E = CFG.n_experts
+    with pytest.raises(binding.DynamoError) as ei:
+        gpu.set_channel_precision_down([5] * E)
+    assert ei.value.status == ERR("ERR_BITS")
+    fresh = binding.DynamoLayer.from_config(CFG, max_tokens=16)
+    with pytest.raises(binding.DynamoError) as ei:
+        fresh.set_channel_precision_down([8] * E)
+    assert ei.value.status == ERR("ERR_STATE")
 
 
 def test_switch_enqueued_between_two_forwards_takes_effect_between_them(lay):
