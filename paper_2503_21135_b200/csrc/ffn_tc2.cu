@@ -63,6 +63,7 @@ static_assert(T2_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 constexpr uint32_t T2_TMEM_COLS = 512;
 constexpr uint32_t T2_COL_A = 256;
 constexpr int T2_NA = 4;                               // A buffers of 64 columns: the dequant warps run ahead of the MMA
+constexpr int T2_LEAD = 2;                             // stages of the next item dequantized before an item's epilogue
 
 struct T2Params {
     const LayerDev* L;
@@ -387,65 +388,85 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
         const uint32_t my_lanes = tbase + ((uint32_t)(32 * q + 16 * asel) << 16);
         bool ok = true, clamped = false;
         uint32_t ic = 0;
-        for (int g = cluster_id; g < total && ok; g += n_clusters, ++ic) {
-            const T2Item w = t2_decode_item<GATEUP>(p, prefix, g, cursor, n_kc, rank);
-            const int bits = w.bits;
-            for (int it = 0; it < w.n_it && ok; ++it, ++gi) {
-                if ((int)(gi & 1) != kh) continue;
-                const int s = gi % T2_NW, ph = (gi / T2_NW) & 1;     // weight slot (= kh: a warp always uses the same one)
-                const int xs = gi % T2_NX, xph = (gi / T2_NX) & 1;   // operand slot
-                const int b = gi % T2_NA, bph = (gi / T2_NA) & 1;
-                const uint8_t* st = wring + (size_t)s * T2_WHALF_MAX;
-                ok = mbar_wait_bounded(&B->full[s], ph, poison, status) &&
-                     mbar_wait_bounded(&B->a_empty[b], bph ^ 1, poison, status);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t a_cols = my_lanes + T2_COL_A + 64 * b;
-                if (it < n_kc) {
-                    switch (bits) {
-                        case 2: t2_dequant_half<2>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<2>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
-                        case 3: t2_dequant_half<3>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<3>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
-                        case 4: t2_dequant_half<4>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<4>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
-                        case 6: t2_dequant_half<6>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<6>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
-                        default: t2_dequant_half<8>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<8>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
-                    }
-                } else {
-                    // cached-channel stage: fp16 tiles [pool column][256 rows] -> A fragments -> tensor memory;
-                    const int mi = lane >> 3, r = lane & 7;
-                    for (int j = 0; j < 2; ++j) {
-                        uint32_t af[4];
-                        const uint32_t addr = smem_u32(st + (j * 16 + (mi >> 1) * 8 + r) * POOL_TILE_PITCH +
-                                                       (16 * atom_g + (mi & 1) * 8) * 2);
-                        asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                                     : "=r"(af[0]), "=r"(af[1]), "=r"(af[2]), "=r"(af[3])
-                                     : "r"(addr));
-                        tc_st_x1(a_cols + 8 * j, af[0], af[2], af[1], af[3]);
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&B->empty[s]);  // the tiles are in registers / tensor memory
+        // One visit: stage `it` of item w, whose running stage number (ring slots, barrier phases) is gis.
+        auto visit = [&](const T2Item& w, int it, uint32_t gis) -> bool {
+            const int s = gis % T2_NW, ph = (gis / T2_NW) & 1;     // weight slot (= kh: a warp always uses the same one)
+            const int xs = gis % T2_NX, xph = (gis / T2_NX) & 1;   // operand slot
+            const int b = gis % T2_NA, bph = (gis / T2_NA) & 1;
+            const uint8_t* st = wring + (size_t)s * T2_WHALF_MAX;
+            if (!(mbar_wait_bounded(&B->full[s], ph, poison, status) &&
+                  mbar_wait_bounded(&B->a_empty[b], bph ^ 1, poison, status)))
+                return false;
+            tc_fence_after();
+            const uint32_t a_cols = my_lanes + T2_COL_A + 64 * b;
+            if (it < n_kc) {
+                switch (w.bits) {
+                    case 2: t2_dequant_half<2>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<2>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
+                    case 3: t2_dequant_half<3>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<3>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
+                    case 4: t2_dequant_half<4>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<4>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
+                    case 6: t2_dequant_half<6>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<6>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
+                    default: t2_dequant_half<8>(st, a_cols, a_l, 0, lane, G, nullptr); t2_dequant_half<8>(st, a_cols, a_l, 1, lane, G, &B->empty[s]); break;
                 }
-                tc_wait_st();
-                // the arrive below also vouches for this CTA's half of the operand tile (the MMA reads both halves)
-                ok = mbar_wait_bounded(&B->fullx[xs], xph, poison, status);
-                if (!ok) break;
-                tc_fence_before();
+            } else {
+                // cached-channel stage: fp16 tiles [pool column][256 rows] -> A fragments -> tensor memory;
+                const int mi = lane >> 3, r = lane & 7;
+                for (int j = 0; j < 2; ++j) {
+                    uint32_t af[4];
+                    const uint32_t addr = smem_u32(st + (j * 16 + (mi >> 1) * 8 + r) * POOL_TILE_PITCH +
+                                                   (16 * atom_g + (mi & 1) * 8) * 2);
+                    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                                 : "=r"(af[0]), "=r"(af[1]), "=r"(af[2]), "=r"(af[3])
+                                 : "r"(addr));
+                    tc_st_x1(a_cols + 8 * j, af[0], af[2], af[1], af[3]);
+                }
                 __syncwarp();
-                if (lane == 0) {  // the barrier lives in the leader: a plain arrive there, a remote one from the peer
-                    if (rank == 0) mbar_arrive(&B->a_full[b]);
-                    else mbar_arrive_remote(&B->a_full[b], 0);
-                }
+                if (lane == 0) mbar_arrive(&B->empty[s]);  // the tiles are in registers / tensor memory
+            }
+            tc_wait_st();
+            // the arrive below also vouches for this CTA's half of the operand tile (the MMA reads both halves)
+            if (!mbar_wait_bounded(&B->fullx[xs], xph, poison, status)) return false;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {  // the barrier lives in the leader: a plain arrive there, a remote one from the peer
+                if (rank == 0) mbar_arrive(&B->a_full[b]);
+                else mbar_arrive_remote(&B->a_full[b], 0);
+            }
+            return true;
+        };
+        // The first T2_LEAD stages of the NEXT item are dequantized before this item's epilogue: their A buffers come
+        // free while the last MMAs of this item still run, so when the epilogue hands the accumulators back the MMA
+        // warp finds two stages ready instead of waiting for a whole dequantization visit.
+        T2Item w = t2_decode_item<GATEUP>(p, prefix, cluster_id, cursor, n_kc, rank);
+        int lead_done = 0;                       // stages of w already dequantized (as the previous item's lead)
+        for (int g = cluster_id; g < total && ok; g += n_clusters, ++ic) {
+            const int bits = w.bits;
+            for (int it = lead_done; it < w.n_it && ok; ++it)
+                if ((int)((gi + it) & 1) == kh) ok = visit(w, it, gi + it);
+            gi += w.n_it;
+            T2Item nx = w;
+            lead_done = 0;
+            if (g + n_clusters < total) {
+                nx = t2_decode_item<GATEUP>(p, prefix, g + n_clusters, cursor, n_kc, rank);
+                lead_done = nx.n_it < T2_LEAD ? nx.n_it : T2_LEAD;
+                for (int it = 0; it < lead_done && ok; ++it)
+                    if ((int)((gi + it) & 1) == kh) ok = visit(nx, it, gi + it);
             }
             if (ok) ok = mbar_wait_bounded(&B->d_full, ic & 1, poison, status);
             tc_fence_after();
             if (ok) {
                 // this warp: its atom's 16 accumulator rows x the tokens [128*kh, 128*kh + 128) of the tile
                 const float scl = __uint_as_float((uint32_t)(127 + x_scale_exp(bits, 8 * atom_g + gid)) << 23);
+                // (the next 32 columns are requested before these are processed)
+                uint32_t rr[2][16];
+                const int ncb = min(4, (w.n_mma - 128 * kh + 31) >> 5);
+                if (ncb > 0) tc_ld_x4(my_lanes + 128 * kh, rr[0]);
+#pragma unroll
                 for (int cb = 0; cb < 4; ++cb) {
                     const int col0 = 128 * kh + 32 * cb;
-                    if (col0 >= w.n_mma) break;
-                    uint32_t r[16];
-                    tc_ld_x4(my_lanes + col0, r);
+                    if (cb >= ncb) break;
                     tc_wait_ld();
+                    if (cb + 1 < ncb) tc_ld_x4(my_lanes + col0 + 32, rr[(cb + 1) & 1]);
+                    const uint32_t (&r)[16] = rr[cb & 1];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         if constexpr (GATEUP) {
@@ -489,6 +510,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) ffn_tc2_kernel(const T2Params p
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_remote(&B->d_empty, 0);
+            w = nx;
         }
         if (clamped) atomicOr(status, STATUS_RANGE);
     }
