@@ -251,14 +251,20 @@ dynamo_status dynamo_set_channel_precision(dynamo_ctx* ctx, const int32_t* hi_bi
  * dynamo_select_significant: per expert with base bits < 8 the n_select (<= max_sig, <= P) cached channels with
  *   the largest A, ties -> lower channel index, become the significant set (slot order = rank order); 8-bit
  *   experts get the empty set.  The tables are rewritten by a device kernel exactly as dynamo_set_channel_switch
- *   would write them; the call then SYNCHRONISES the stream to bring the chosen sets back (host mirror, and
- *   sig_idx_out host [E, max_sig] padded with -1 / sig_cnt_out host [E] if not NULL).  reset != 0 zeroes A.
+ *   would write them, in stream order.  With sig_idx_out and sig_cnt_out both NULL the call does not wait: the
+ *   chosen sets travel to a pinned host buffer behind the kernel and the library reads them when the host next
+ *   needs them (dynamo_sync_sets, dynamo_expert_stream_bytes, a later switch).  With an output pointer given
+ *   (sig_idx_out host [E, max_sig] padded with -1, sig_cnt_out host [E]) the call waits for that copy and fills
+ *   them, as dynamo_sync_sets would.  reset != 0 zeroes A.  The first call allocates the pinned buffer and an event.
+ * dynamo_sync_sets: waits for the sets of the last dynamo_select_significant (if still on their way) and returns
+ *   the sets now installed, whoever installed them; either pointer may be NULL.
  * Errors: NULL ctx -> ERR_NULL; before pack -> ERR_STATE; n_select out of range or a pool too large to rank in
  * shared memory (P > 12288) -> ERR_SHAPE. */
 dynamo_status dynamo_set_stats_collection(dynamo_ctx* ctx, int32_t on);
 dynamo_status dynamo_get_channel_stats(dynamo_ctx* ctx, float* stats_out, void* stream);
 dynamo_status dynamo_select_significant(dynamo_ctx* ctx, int32_t n_select, int32_t reset, int32_t* sig_idx_out,
                                         int32_t* sig_cnt_out, void* stream);
+dynamo_status dynamo_sync_sets(dynamo_ctx* ctx, int32_t* sig_idx_out, int32_t* sig_cnt_out);
 
 /* Significant channels on the d_ff side (Section IV-B applied to the second projection: the input channels of
  * W_down are the hidden units).  Optional; a layer that never calls these pays nothing.

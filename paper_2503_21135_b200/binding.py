@@ -35,7 +35,7 @@ EXPORTED = ["dynamo_create", "dynamo_destroy", "dynamo_arena_bytes", "dynamo_pac
             "dynamo_poll_status", "dynamo_set_profile_events", "dynamo_set_tc_min_rows", "dynamo_set_operand_dtype", "dynamo_set_stats_collection", "dynamo_set_channel_precision", "dynamo_assign_bits",
             "dynamo_down_cache_bytes", "dynamo_pack_down_cache", "dynamo_set_channel_switch_down",
             "dynamo_set_channel_precision_down",
-            "dynamo_get_channel_stats", "dynamo_select_significant", "dynamo_route_permute_static",
+            "dynamo_get_channel_stats", "dynamo_select_significant", "dynamo_sync_sets", "dynamo_route_permute_static",
             "dynamo_debug_expire_wait", "dynamo_debug_check_guards",
             "dynamo_kernel_launches", "dynamo_status_str"]
 
@@ -94,6 +94,7 @@ def load():
                                          ctypes.c_double, i32p, i32p, f64p, f64p, i32p]
         L.dynamo_get_channel_stats.argtypes = [vp, vp, vp]
         L.dynamo_select_significant.argtypes = [vp, i32, i32, i32p, i32p, vp]
+        L.dynamo_sync_sets.argtypes = [vp, i32p, i32p]
         L.dynamo_route_permute_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
         L.dynamo_debug_expire_wait.argtypes = [vp, ctypes.c_int64, vp]
         L.dynamo_debug_check_guards.argtypes = [vp, ctypes.POINTER(ctypes.c_int64), vp]
@@ -408,13 +409,26 @@ class DynamoLayer:
         _check(load().dynamo_get_channel_stats(self.ctx, out.data_ptr(), _stream()), "dynamo_get_channel_stats")
         return out
 
-    def select_significant(self, n_select: int, reset: bool = True):
-        """Install, per expert, the n_select cached channels with the largest statistics; returns the sets."""
+    def select_significant(self, n_select: int, reset: bool = True, wait: bool = True):
+        """Install, per expert, the n_select cached channels with the largest statistics.  wait=True returns the sets;
+        wait=False only enqueues the selection (fetch the sets later with sync_sets)."""
+        if not wait:
+            _check(load().dynamo_select_significant(self.ctx, n_select, int(bool(reset)), None, None, _stream()),
+                   "dynamo_select_significant")
+            return None
         E, S = self.desc.n_experts, self.desc.max_sig
         idx = np.full((E, max(S, 1)), -1, dtype=np.int32)
         cnt = np.zeros((E,), dtype=np.int32)
         _check(load().dynamo_select_significant(self.ctx, n_select, int(bool(reset)), _i32p(idx), _i32p(cnt), _stream()),
                "dynamo_select_significant")
+        return [idx[e, : cnt[e]].copy() for e in range(E)]
+
+    def sync_sets(self):
+        """The significant sets now installed (waits for a selection still on its way)."""
+        E, S = self.desc.n_experts, self.desc.max_sig
+        idx = np.full((E, max(S, 1)), -1, dtype=np.int32)
+        cnt = np.zeros((E,), dtype=np.int32)
+        _check(load().dynamo_sync_sets(self.ctx, _i32p(idx), _i32p(cnt)), "dynamo_sync_sets")
         return [idx[e, : cnt[e]].copy() for e in range(E)]
 
     def set_profile_events(self, events=None):

@@ -262,6 +262,18 @@ struct dynamo_ctx {
     int64_t launches = 0;
     cudaEvent_t prof_ev[3] = {nullptr, nullptr, nullptr};  // optional: before gate/up, after gate/up, after down
     std::vector<int32_t> upload;                 // scratch for switch uploads
+    // Sets chosen on the device (dynamo_select_significant) come back through a pinned buffer and an event; the host
+    // mirror `sig` is brought up to date by the next call that reads it.
+    int32_t* mirror_host = nullptr;              // pinned [E][S_pad]
+    cudaEvent_t mirror_ev = nullptr;
+    bool mirror_pending = false;
+    ~dynamo_ctx() {
+        if (mirror_ev) {
+            cudaEventSynchronize(mirror_ev);
+            cudaEventDestroy(mirror_ev);
+        }
+        if (mirror_host) cudaFreeHost(mirror_host);
+    }
 };
 
 namespace {
@@ -430,6 +442,36 @@ dynamo_status dynamo_set_channel_precision(dynamo_ctx* ctx, const int32_t* hi_bi
     return DYNAMO_OK;
 }
 
+// Wait for the sets the device chose last (if any are still on their way) and update the host mirror.
+static dynamo_status sync_mirror(dynamo_ctx* ctx) {
+    if (!ctx->mirror_pending) return DYNAMO_OK;
+    CUDA_TRY(cudaEventSynchronize(ctx->mirror_ev));
+    const int E = ctx->D.n_experts, S_pad = s_pad_of(ctx->D);
+    for (int e = 0; e < E; ++e) {
+        std::vector<int32_t>& lst = ctx->sig[e];
+        lst.clear();
+        for (int j = 0; j < S_pad && ctx->mirror_host[(size_t)e * S_pad + j] >= 0; ++j)
+            lst.push_back(ctx->mirror_host[(size_t)e * S_pad + j]);
+    }
+    ctx->mirror_pending = false;
+    return DYNAMO_OK;
+}
+
+dynamo_status dynamo_sync_sets(dynamo_ctx* ctx, int32_t* sig_idx_out, int32_t* sig_cnt_out) {
+    if (!ctx) return DYNAMO_ERR_NULL;
+    if (!ctx->packed) return DYNAMO_ERR_STATE;
+    dynamo_status s = sync_mirror(ctx);
+    if (s != DYNAMO_OK) return s;
+    const dynamo_layer_desc& D = ctx->D;
+    for (int e = 0; e < D.n_experts; ++e) {
+        const std::vector<int32_t>& lst = ctx->sig[e];
+        if (sig_cnt_out) sig_cnt_out[e] = (int32_t)lst.size();
+        if (sig_idx_out)
+            for (int j = 0; j < D.max_sig; ++j) sig_idx_out[(size_t)e * D.max_sig + j] = j < (int)lst.size() ? lst[j] : -1;
+    }
+    return DYNAMO_OK;
+}
+
 dynamo_status dynamo_set_stats_collection(dynamo_ctx* ctx, int32_t on) {
     if (!ctx) return DYNAMO_ERR_NULL;
     ctx->collect_stats = on ? 1 : 0;
@@ -455,22 +497,22 @@ dynamo_status dynamo_select_significant(dynamo_ctx* ctx, int32_t n_select, int32
     if ((size_t)D.cache_size * 4 > 48 * 1024) return DYNAMO_ERR_SHAPE;  // the ranking keeps a pool's statistics in shared memory
     cudaStream_t st = (cudaStream_t)stream;
     const int E = D.n_experts, S_pad = s_pad_of(D);
+    dynamo_status ms = sync_mirror(ctx);   // the pinned buffer is about to be reused
+    if (ms != DYNAMO_OK) return ms;
+    if (!ctx->mirror_host) {
+        CUDA_TRY(cudaMallocHost((void**)&ctx->mirror_host, (size_t)E * S_pad * 4));
+        CUDA_TRY(cudaEventCreateWithFlags(&ctx->mirror_ev, cudaEventDisableTiming));
+    }
     int32_t* chosen = (int32_t*)(ctx->ws + ctx->W.stage_switch);
     CUDA_TRY(launch_select((const LayerDev*)ctx->arena, (float*)(ctx->arena + ctx->A.stats), E, D.cache_size, n_select,
                            reset ? 1 : 0, chosen, st));
     ctx->launches += 1;
-    // the host mirror of the sets (stream bytes, exports, later validation) follows the device's choice
-    std::vector<int32_t> host((size_t)E * S_pad);
-    CUDA_TRY(cudaMemcpyAsync(host.data(), chosen, host.size() * 4, cudaMemcpyDeviceToHost, st));
-    CUDA_TRY(cudaStreamSynchronize(st));
-    for (int e = 0; e < E; ++e) {
-        std::vector<int32_t>& lst = ctx->sig[e];
-        lst.clear();
-        for (int j = 0; j < S_pad && host[(size_t)e * S_pad + j] >= 0; ++j) lst.push_back(host[(size_t)e * S_pad + j]);
-        if (sig_cnt_out) sig_cnt_out[e] = (int32_t)lst.size();
-        if (sig_idx_out)
-            for (int j = 0; j < D.max_sig; ++j) sig_idx_out[(size_t)e * D.max_sig + j] = j < (int)lst.size() ? lst[j] : -1;
-    }
+    // the host mirror of the sets (stream bytes, later switches in requantize mode) follows the device's choice: the
+    // chosen sets travel to a pinned buffer in stream order and are read when the host next needs them
+    CUDA_TRY(cudaMemcpyAsync(ctx->mirror_host, chosen, (size_t)E * S_pad * 4, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaEventRecord(ctx->mirror_ev, st));
+    ctx->mirror_pending = true;
+    if (sig_idx_out || sig_cnt_out) return dynamo_sync_sets(ctx, sig_idx_out, sig_cnt_out);
     return DYNAMO_OK;
 }
 
@@ -512,6 +554,10 @@ dynamo_status dynamo_pack_experts(dynamo_ctx* ctx, const void* w_gate, const voi
     ctx->down_arena = nullptr;  // a d_ff-side cache belongs to the previous packing
     ctx->down_active = 0;
     ctx->cache_idx.assign(cache_idx, cache_idx + (size_t)D.n_experts * P);
+    if (ctx->mirror_pending) {  // sets chosen for the previous packing: let the copy land, then drop them
+        CUDA_TRY(cudaEventSynchronize(ctx->mirror_ev));
+        ctx->mirror_pending = false;
+    }
     ctx->sig.assign(D.n_experts, {});
 
     CUDA_TRY(cudaMemsetAsync(ctx->arena, 0, A.total, st));
@@ -597,6 +643,10 @@ dynamo_status dynamo_set_channel_switch_many(dynamo_ctx* const* ctxs, int32_t n_
         if (!ctxs[l]) return DYNAMO_ERR_NULL;
         if (!ctxs[l]->packed) return DYNAMO_ERR_STATE;
         if (std::memcmp(&ctxs[l]->D, &ctxs[0]->D, sizeof(dynamo_layer_desc)) != 0) return DYNAMO_ERR_SHAPE;
+    }
+    for (int l = 0; l < n_layers; ++l) {  // sets the device chose earlier enter the host mirror first
+        dynamo_status ms = sync_mirror(ctxs[l]);
+        if (ms != DYNAMO_OK) return ms;
     }
     dynamo_ctx* c0 = ctxs[0];
     const dynamo_layer_desc& D = c0->D;
@@ -949,6 +999,8 @@ dynamo_status dynamo_expert_stream_bytes(dynamo_ctx* ctx, int32_t expert, size_t
     const dynamo_layer_desc& D = ctx->D;
     if (expert < 0 || expert >= D.n_experts + D.n_shared) return DYNAMO_ERR_SHAPE;
     const size_t d = D.d_model, f = D.d_ff;
+    dynamo_status ms = sync_mirror(ctx);
+    if (ms != DYNAMO_OK) return ms;
     const size_t blocks = (2 * f / RB) * (d / KC) + (d / RB) * (f / KC);
     size_t b = blocks * (size_t)block_bytes(ctx->bits[expert], D.group_size);
     if (expert < D.n_experts && ctx->bits[expert] < HI_BITS) b += 2 * f * ctx->sig[expert].size() * 2;

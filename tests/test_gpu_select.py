@@ -123,6 +123,36 @@ def test_selection_tracks_a_change_of_the_data(tiny):
     gpu.set_channel_switch(tiny["sets"])
 
 
+def test_selection_enqueued_without_waiting_takes_effect_in_stream_order(tiny):
+    """forward, select (no wait), forward, with no host synchronisation in between: the second forward runs on the
+    selected sets; the sets reach the host afterwards through dynamo_sync_sets."""
+    gpu = tiny["gpu"]
+    x, lg = wl.activations(CFG, 48, step=33).cuda(), wl.router_logits(CFG, 48, step=33).cuda()
+    gpu.select_significant(0, reset=True)
+    gpu.set_stats_collection(True)
+    gpu.forward(x, lg, binding.F32)
+    gpu.set_stats_collection(False)
+    stats = gpu.channel_stats().clone()
+    torch.cuda.synchronize()
+    y_before = torch.empty((48, CFG.d_model), dtype=torch.float32, device="cuda")
+    y_after = torch.empty_like(y_before)
+    gpu.forward(x, lg, binding.F32, y=y_before)
+    assert gpu.select_significant(6, reset=False, wait=False) is None
+    gpu.forward(x, lg, binding.F32, y=y_after)
+    sets = gpu.sync_sets()
+    torch.cuda.synchronize()
+    ref_sets = oracle.select_significant(stats.cpu().numpy(), tiny["pool"], 6, [int(b) < 8 for b in tiny["bits"][:CFG.n_experts]])
+    for e in range(CFG.n_experts):
+        assert sets[e].tolist() == ref_sets[e].tolist(), e
+    gpu.set_channel_switch([np.array([], np.int32)] * CFG.n_experts)
+    assert torch.equal(gpu.forward(x, lg, binding.F32), y_before)
+    gpu.set_channel_switch(ref_sets)
+    assert torch.equal(gpu.forward(x, lg, binding.F32), y_after)
+    assert not torch.equal(y_before, y_after)
+    assert [s.tolist() for s in gpu.sync_sets()] == [s.tolist() for s in ref_sets]   # whoever installed them
+    gpu.set_channel_switch(tiny["sets"])
+
+
 def test_selection_errors(tiny):
     gpu = tiny["gpu"]
     st = binding.load().dynamo_select_significant(gpu.ctx, CFG.max_sig + 1, 0, None, None, None)
