@@ -41,7 +41,8 @@ cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, in
 cudaError_t setup_ffn_tc2(int n_sms, int* clusters_out);
 cudaError_t launch_ffn_tc2(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int n_experts, int n_clusters,
                            cudaStream_t st);
-cudaError_t launch_stats(const LayerDev* L, const WsDev& ws, const void* x, float* stats, int E, cudaStream_t st);
+cudaError_t launch_stats(const LayerDev* L, const WsDev& ws, const void* x, float* stats, float* part, int32_t* ctr, int E,
+                         int n_slices, cudaStream_t st);
 cudaError_t launch_select(const LayerDev* L, float* stats, int E, int P, int n_sel, int reset, int32_t* chosen,
                           cudaStream_t st);
 cudaError_t launch_expire_wait(int32_t* status, unsigned long long limit_ns, cudaStream_t st);
@@ -68,7 +69,7 @@ constexpr int GUARD_BYTE = 0xC5;
 struct ArenaLayout {
     size_t header = 0;
     std::vector<size_t> w13, w2, s8m8_g, s8m8_u, mm_g, mm_u, q8_g, q8_u, cw_g, cw_u, pool_hi;
-    size_t cache_idx = 0, sig_chan = 0, sig_pool = 0, sig_cnt = 0, sigmask = 0, stats = 0;
+    size_t cache_idx = 0, sig_chan = 0, sig_pool = 0, sig_cnt = 0, sigmask = 0, stats = 0, stats_ctr = 0;
     size_t total = 0;
     std::vector<size_t> guards;  // offsets of the guard blocks
 };
@@ -191,6 +192,7 @@ void arena_layout(const dynamo_layer_desc& D, const int32_t* bits, ArenaLayout& 
     A.sig_cnt = take((size_t)D.n_experts * 4);
     A.sigmask = take((size_t)D.n_experts * (d / 32) * 4);
     A.stats = take((size_t)D.n_experts * ((P + 31) / 32 * 32) * 4);  // activation mass per (expert, cached channel)
+    A.stats_ctr = take((size_t)D.n_experts * 4);                     // arrival counters of the statistics kernel's slices
     A.total = off;
 }
 
@@ -760,7 +762,14 @@ static dynamo_status forward_impl(dynamo_ctx* ctx, const void* x, const float* r
         CUDA_TRY(launch_gather(L, ws, x, st));
     }
     if (ctx->collect_stats) {
-        CUDA_TRY(launch_stats(L, ws, x, (float*)(ctx->arena + ctx->A.stats), D.n_experts, st));
+        // row slices per expert: about two CTAs per SM in all; the partial sums live in the down GEMM's output buffer
+        // (at least 8 * (E + Es) rows of d floats, idle until the down launch), which bounds the slice count
+        const int P_pad = ctx->host_layer.P_pad;
+        int n_slices = std::max(1, std::min(32, (2 * ctx->n_sms + D.n_experts - 1) / D.n_experts));
+        n_slices = std::max(1, std::min(n_slices, 8 * D.d_model / std::max(P_pad, 1)));
+        if ((long long)T * D.top_k <= 16ll * D.n_experts) n_slices = 1;  // a few rows per expert: one pass is shorter
+        CUDA_TRY(launch_stats(L, ws, x, (float*)(ctx->arena + ctx->A.stats), ws.ypart,
+                              (int32_t*)(ctx->arena + ctx->A.stats_ctr), D.n_experts, n_slices, st));
         ctx->launches += 1;
     }
     const bool use_tc = ws.tc_min != 0x7fffffff;                  // experts above 32 rows take the tcgen05 path

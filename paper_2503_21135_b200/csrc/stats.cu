@@ -3,8 +3,9 @@
 //
 // stats  : while forwards run, per routed expert e and cached channel c the activation mass
 //              A[e][c] += sum over the tokens routed to e in this forward of |x[t][c]|
-//          is accumulated in fp32 in a FIXED order (tokens ascending inside a forward, one addition of the
-//          forward's sum to the running total), so the numbers are reproducible bit for bit.
+//          is accumulated in fp32 in a FIXED order (the expert's rows are cut into slices, one CTA each: tokens
+//          ascending inside a slice, slices ascending, one addition of the forward's sum to the running total),
+//          so the numbers are reproducible bit for bit for a given slice count.
 // select : per expert the S cached channels with the largest A (ties -> lower channel index) become the
 //          significant set, in rank order; the index tables and the channel bitmask are rewritten on the
 //          device exactly as a host-driven switch would write them.
@@ -12,24 +13,47 @@
 
 namespace dyn {
 
-// grid (E), 256 threads: thread j walks the expert's rows for cached channel j.
+// grid (E, n_slices), 256 threads: CTA (e, s) walks slice s of the expert's rows, thread j for cached channel j, and
+// leaves its partial sums in `part` [E][n_slices][P_pad] (scratch: the down GEMM's output buffer, not yet in use at
+// this point of a forward); the CTA that finishes last for an expert (a self-resetting counter per expert) adds the
+// slices up in slice order and adds the result to the running total.
 __global__ void __launch_bounds__(256) stats_kernel(const LayerDev* __restrict__ L, WsDev ws,
-                                                    const __nv_bfloat16* __restrict__ x, float* __restrict__ stats) {
+                                                    const __nv_bfloat16* __restrict__ x, float* __restrict__ stats,
+                                                    float* __restrict__ part, int32_t* __restrict__ ctr) {
+    __shared__ int s_last;
     pdl_prologue();
-    const int e = blockIdx.x;
+    const int e = blockIdx.x, s = blockIdx.y, nsl = gridDim.y;
     const int P = L->P, P_pad = L->P_pad, d = L->d;
     const int cnt = ws.counts[e], row0 = ws.off_pad[e];
-    if (cnt == 0) return;
+    if (cnt == 0) return;  // every slice of the expert leaves: its counter stays at zero
+    const int len = (cnt + nsl - 1) / nsl;
+    const int r0 = min(cnt, s * len), r1 = min(cnt, r0 + len);
     const int32_t* ci = L->cache_idx + (long long)e * P;
+    float* mine = part + ((long long)e * nsl + s) * P_pad;
     for (int j = threadIdx.x; j < P; j += blockDim.x) {
         const int ch = ci[j];
         float sum = 0.f;
-        for (int r = 0; r < cnt; ++r) {
+#pragma unroll 4
+        for (int r = r0; r < r1; ++r) {
             const int t = ws.row_token[row0 + r];
             sum += fabsf(__bfloat162float(x[(long long)t * d + ch]));
         }
-        stats[(long long)e * P_pad + j] += sum;
+        if (nsl == 1) stats[(long long)e * P_pad + j] += sum;   // a single slice: no second pass
+        else mine[j] = sum;
     }
+    if (nsl == 1) return;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(&ctr[e], 1) == nsl - 1) ? 1 : 0;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    for (int j = threadIdx.x; j < P; j += blockDim.x) {
+        float tot = 0.f;
+        for (int q = 0; q < nsl; ++q) tot += __ldcg(part + ((long long)e * nsl + q) * P_pad + j);
+        stats[(long long)e * P_pad + j] += tot;
+    }
+    if (threadIdx.x == 0) ctr[e] = 0;
 }
 
 // grid (E), 256 threads.  rank(j) = number of cached channels that beat j (larger A, or equal A and lower channel
@@ -67,8 +91,11 @@ __global__ void __launch_bounds__(256) select_kernel(const LayerDev* __restrict_
     if (threadIdx.x == 0) L->sig_cnt[e] = cnt;
 }
 
-cudaError_t launch_stats(const LayerDev* L, const WsDev& ws, const void* x, float* stats, int E, cudaStream_t st) {
-    return launch_pdl(stats_kernel, dim3((unsigned)E), dim3(256), 0, st, L, ws, (const __nv_bfloat16*)x, stats);
+// part: scratch of E * n_slices * P_pad floats; ctr: E zero-initialised counters (left at zero).
+cudaError_t launch_stats(const LayerDev* L, const WsDev& ws, const void* x, float* stats, float* part, int32_t* ctr, int E,
+                         int n_slices, cudaStream_t st) {
+    return launch_pdl(stats_kernel, dim3((unsigned)E, (unsigned)n_slices), dim3(256), 0, st, L, ws,
+                      (const __nv_bfloat16*)x, stats, part, ctr);
 }
 
 cudaError_t launch_select(const LayerDev* L, float* stats, int E, int P, int n_sel, int reset, int32_t* chosen,
