@@ -267,7 +267,8 @@ __global__ void __launch_bounds__(1024) scan_kernel(WsDev ws, int E, int Es, int
 
 // One CTA per physical row; warp w converts chunks w, w+8, ...  (Eight rows per CTA with one warp per row, so that
 // the chain of dependent loads that finds a row's expert is paid once per eight rows, measured slower: +18 us on the
-// 64-token step, nothing gained at 4096 tokens.)  The fp16 activations are stored
+// 64-token step, nothing gained at 4096 tokens; staging a token's pair rows and weights in shared memory in the
+// combine kernel measured no gain either.)  The fp16 activations are stored
 // multiplied by 2^x_scale_exp(bits of the row's expert, k) so that the FFN kernels can use packed codes
 // in place; the per-group sums are of the unscaled fp16 values.
 __device__ __forceinline__ void gather_row(const LayerDev* __restrict__ L, const WsDev& ws,
@@ -496,41 +497,23 @@ __global__ void __launch_bounds__(256) combine_kernel(WsDev ws, int d, int k, in
                                                       int y_f32, long long split_stride) {
     pdl_prologue();
     if (*ws.status & STATUS_TIMEOUT) return;  // the FFN kernels started nothing: leave y alone
-    // row, weight and K-split count of the token's pairs: found once per CTA (a chain of three dependent loads per
-    // pair), so that the threads' loads of the partial outputs below are all independent
-    __shared__ int s_r[32], s_ns[32];
-    __shared__ float s_w[32];
     const int t = blockIdx.x;
     const int kk = k + Es;
     const int c = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int j0 = 0; j0 < kk; j0 += 32) {
-        const int nj = min(32, kk - j0);
-        if (j0) __syncthreads();
-        if ((int)threadIdx.x < nj) {
-            const int j = j0 + threadIdx.x;
-            const int r = ws.pos[t * kk + j];
-            s_r[threadIdx.x] = r;
-            s_w[threadIdx.x] = (j < k) ? ws.topk_w[t * k + j] : 1.0f;
-            s_ns[threadIdx.x] = (ws.counts[ws.row_expert[r]] > ws.tc_min) ? 1 : ws.ksplit;  // the tensor-core path does not split K
-        }
-        __syncthreads();
-        if (c < d) {
-#pragma unroll 4
-            for (int jj = 0; jj < nj; ++jj) {
-                const int r = s_r[jj], ns = s_ns[jj];
-                const float w = s_w[jj];
-                float s[4] = {0.f, 0.f, 0.f, 0.f};
-                for (int sp = 0; sp < ns; ++sp) {
-                    const float4 v = *reinterpret_cast<const float4*>(ws.ypart + sp * split_stride + (long long)r * d + c);
-                    s[0] += v.x; s[1] += v.y; s[2] += v.z; s[3] += v.w;
-                }
-#pragma unroll
-                for (int i = 0; i < 4; ++i) acc[i] = fmaf(w, s[i], acc[i]);
-            }
-        }
-    }
     if (c >= d) return;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int j = 0; j < kk; ++j) {
+        const int r = ws.pos[t * kk + j];
+        const float w = (j < k) ? ws.topk_w[t * k + j] : 1.0f;
+        float s[4] = {0.f, 0.f, 0.f, 0.f};
+        const int ns = (ws.counts[ws.row_expert[r]] > ws.tc_min) ? 1 : ws.ksplit;  // the tensor-core path does not split K
+        for (int sp = 0; sp < ns; ++sp) {
+            const float4 v = *reinterpret_cast<const float4*>(ws.ypart + sp * split_stride + (long long)r * d + c);
+            s[0] += v.x; s[1] += v.y; s[2] += v.z; s[3] += v.w;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[i] = fmaf(w, s[i], acc[i]);
+    }
     if (y_f32) {
         *reinterpret_cast<float4*>((float*)y + (long long)t * d + c) = make_float4(acc[0], acc[1], acc[2], acc[3]);
     } else {
