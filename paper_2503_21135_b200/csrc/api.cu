@@ -37,7 +37,7 @@ cudaError_t launch_front(const LayerDev* L, const WsDev& ws, const void* x, cons
 cudaError_t launch_combine(const WsDev& ws, int d, int k, int Es, void* y, int y_f32, long long split_stride,
                            cudaStream_t st);
 cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int ksplit, int n_experts,
-                              long long split_stride, int max_rows, int n_sms, cudaStream_t st);
+                              long long split_stride, int max_rows, int n_sms, int G, cudaStream_t st);
 cudaError_t setup_ffn_tc2(int n_sms, int* clusters_out);
 cudaError_t launch_ffn_tc2(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int n_experts, int n_clusters,
                            cudaStream_t st);
@@ -776,10 +776,12 @@ static dynamo_status forward_impl(dynamo_ctx* ctx, const void* x, const float* r
     const long long split_stride = (long long)ws.Rpad * D.d_model;  // partials of one K split: [Rpad][d]
     if (ctx->prof_ev[0]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[0], st));
     const int max_rows = use_tc ? std::min(T, ctx->tc_min_rows) : T;  // rows one expert can have on the streaming path
-    CUDA_TRY(launch_ffn_stream(L, ws, 1, ctx->host_layer.n_rb13, 1, n, split_stride, max_rows, ctx->n_sms, st));
+    CUDA_TRY(launch_ffn_stream(L, ws, 1, ctx->host_layer.n_rb13, 1, n, split_stride, max_rows, ctx->n_sms,
+                               D.group_size, st));
     if (use_tc) CUDA_TRY(launch_ffn_tc2(L, ws, 1, ctx->host_layer.n_rb13, n, ctx->tc2_clusters[1], st));
     if (ctx->prof_ev[1]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[1], st));
-    CUDA_TRY(launch_ffn_stream(L, ws, 0, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, max_rows, ctx->n_sms, st));
+    CUDA_TRY(launch_ffn_stream(L, ws, 0, ctx->host_layer.n_rb2, ws.ksplit, n, split_stride, max_rows, ctx->n_sms,
+                               D.group_size, st));
     if (use_tc) CUDA_TRY(launch_ffn_tc2(L, ws, 0, ctx->host_layer.n_rb2, n, ctx->tc2_clusters[0], st));
     if (ctx->prof_ev[2]) CUDA_TRY(cudaEventRecord(ctx->prof_ev[2], st));
     if (ctx->down_active) {  // significant hidden units: add what their 8-bit columns of W_down change

@@ -96,7 +96,7 @@ __device__ __forceinline__ void mma16816_z(float (&d)[4], const uint32_t (&a)[4]
 
 // Consumer side of one work item.  `stage_it` is the CTA-wide ring position, `item_idx` the number of
 // items this CTA has finished (parity of the epilogue barrier / h tile).
-template <int BITS, int NT8, bool GATEUP>
+template <int BITS, int NT8, bool GATEUP, int G>
 __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uint8_t* stages, uint8_t* htiles,
                                              const Item& im, int& stage_it, int item_idx, bool& clamped) {
     constexpr int NS = MAX_STAGES;
@@ -105,11 +105,10 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gid = lane >> 2, tid4 = lane & 3;
     const int atom0 = warp * APW;
-    const int G = L->G;
     const int K = GATEUP ? L->d : L->f;
     const int n_kc = K / KC;
-    const int blk_bytes = ex.blk_bytes;
     constexpr int code_bytes = 4096 * BITS;
+    constexpr int blk_bytes = code_bytes + RB * (KC / G) * 4;   // = block_bytes(BITS, G), the expert's blk_bytes
     int kc0 = 0, kc1 = n_kc;
     if (!GATEUP) {
         kc0 = (int)(((long long)im.split * n_kc) / p.ksplit);
@@ -129,7 +128,7 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
 
     // exact power of two that undoes the operand scaling: codes enter as q*2^(o-24), activations as x*2^(bias-o)
     const float unscale = __uint_as_float((uint32_t)(127 + 24 - x_scale_bias(BITS)) << 23);
-    const int ngrp = KC / G;
+    constexpr int ngrp = KC / G;
 
     for (int kc = kc0; kc < kc1; ++kc, ++stage_it) {
         const int s = stage_it % NS, ph = (stage_it / NS) & 1;
@@ -296,20 +295,20 @@ __device__ __forceinline__ bool consume_item(const FfnParams& p, FfnSmem* S, uin
 
 // MAXNT8: most 8-token tiles an item can have in this launch (the host knows the token count): the small
 // variants need fewer registers and run three CTAs per SM.
-template <int BITS, bool GATEUP, int MAXNT8>
+template <int BITS, bool GATEUP, int MAXNT8, int G>
 __device__ __forceinline__ bool consume_dispatch(const FfnParams& p, FfnSmem* S, uint8_t* stages, uint8_t* htiles,
                                                  const Item& im, int& stage_it, int item_idx, bool& clamped) {
     const int nt8 = (im.nvalid + 7) >> 3;
-    if (MAXNT8 == 1 || nt8 == 1) return consume_item<BITS, 1, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx, clamped);
+    if (MAXNT8 == 1 || nt8 == 1) return consume_item<BITS, 1, GATEUP, G>(p, S, stages, htiles, im, stage_it, item_idx, clamped);
     if constexpr (MAXNT8 >= 2) {
         if (MAXNT8 == 2 || nt8 == 2)
-            return consume_item<BITS, 2, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx, clamped);
+            return consume_item<BITS, 2, GATEUP, G>(p, S, stages, htiles, im, stage_it, item_idx, clamped);
     }
-    if constexpr (MAXNT8 >= 3) return consume_item<BITS, 3, GATEUP>(p, S, stages, htiles, im, stage_it, item_idx, clamped);
+    if constexpr (MAXNT8 >= 3) return consume_item<BITS, 3, GATEUP, G>(p, S, stages, htiles, im, stage_it, item_idx, clamped);
     return false;
 }
 
-template <bool GATEUP, int MAXNT8>
+template <bool GATEUP, int MAXNT8, int G>
 __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2) ffn_stream_kernel(const FfnParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     pdl_prologue();
@@ -341,7 +340,6 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
     }
     __syncthreads();
     const int n_items = S->n_items;
-    const int G = L->G;
     volatile int* poison = &S->poison;
 
     if (warp == CONSUMER_WARPS) {
@@ -466,7 +464,6 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
     // ---------------- consumer warps ----------------
     int stage_it = 0, y = 0, item_idx = 0;
     bool clamped = false;
-    (void)G;
     const bool all_static = n_items <= (int)gridDim.x;
     for (;; ++item_idx) {
         if (all_static && (item_idx > 0 || (int)blockIdx.x >= n_items)) break;
@@ -481,11 +478,11 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
         const Item im = decode_item(p, S, g, y);
         bool ok;
         switch (L->ex[im.e].bits) {
-            case 2: ok = consume_dispatch<2, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
-            case 3: ok = consume_dispatch<3, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
-            case 4: ok = consume_dispatch<4, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
-            case 6: ok = consume_dispatch<6, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
-            default: ok = consume_dispatch<8, GATEUP, MAXNT8>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
+            case 2: ok = consume_dispatch<2, GATEUP, MAXNT8, G>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
+            case 3: ok = consume_dispatch<3, GATEUP, MAXNT8, G>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
+            case 4: ok = consume_dispatch<4, GATEUP, MAXNT8, G>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
+            case 6: ok = consume_dispatch<6, GATEUP, MAXNT8, G>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
+            default: ok = consume_dispatch<8, GATEUP, MAXNT8, G>(p, S, stages, htiles, im, stage_it, item_idx, clamped); break;
         }
         if (!ok) {  // poisoned: the status word says so; keep arriving so that nobody waits on this warp forever
             if (GATEUP && lane == 0) mbar_arrive(&S->done);
@@ -495,19 +492,24 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
     if (clamped) atomicOr(p.ws.status, STATUS_RANGE);
 }
 
-template <bool GATEUP, int MAXNT8>
-static cudaError_t launch_one(const FfnParams& p, int n_ctas, cudaStream_t st) {
-    cudaError_t err = cudaFuncSetAttribute(ffn_stream_kernel<GATEUP, MAXNT8>,
+template <bool GATEUP, int MAXNT8, int G>
+static cudaError_t launch_one_g(const FfnParams& p, int n_ctas, cudaStream_t st) {
+    cudaError_t err = cudaFuncSetAttribute(ffn_stream_kernel<GATEUP, MAXNT8, G>,
                                            cudaFuncAttributeMaxDynamicSharedMemorySize, p.smem_bytes);
     if (err != cudaSuccess) return err;
-    return launch_pdl(ffn_stream_kernel<GATEUP, MAXNT8>, dim3((unsigned)n_ctas), dim3(FFN_THREADS), (size_t)p.smem_bytes,
-                      st, p);
+    return launch_pdl(ffn_stream_kernel<GATEUP, MAXNT8, G>, dim3((unsigned)n_ctas), dim3(FFN_THREADS),
+                      (size_t)p.smem_bytes, st, p);
+}
+// The group size (64 or 128) is a template parameter: the group bookkeeping of the inner loop folds away.
+template <bool GATEUP, int MAXNT8>
+static cudaError_t launch_one(const FfnParams& p, int n_ctas, int G, cudaStream_t st) {
+    return G == 64 ? launch_one_g<GATEUP, MAXNT8, 64>(p, n_ctas, st) : launch_one_g<GATEUP, MAXNT8, 128>(p, n_ctas, st);
 }
 
 // max_rows: upper bound of the rows one expert can have in this forward (selects the kernel variant);
 // n_sms: SM count (the persistent grid is 2 or 3 CTAs per SM).
 cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, int n_rb, int ksplit, int n_experts,
-                              long long split_stride, int max_rows, int n_sms, cudaStream_t st) {
+                              long long split_stride, int max_rows, int n_sms, int G, cudaStream_t st) {
     // three CTAs per SM pay off once every CTA has several items to walk; at 1-3 tokens a CTA sees one or two
     const bool small = max_rows >= 4 && max_rows <= 16;
     const bool three = small && APW == 2;
@@ -525,9 +527,9 @@ cudaError_t launch_ffn_stream(const LayerDev* L, const WsDev& ws, int gateup, in
     p.n_rb = n_rb;
     p.n_experts = n_experts;
     p.work_ctr = ws.status + (gateup ? 4 : 5);
-    if (small && max_rows <= 8) return gateup ? launch_one<true, 1>(p, n_ctas, st) : launch_one<false, 1>(p, n_ctas, st);
-    if (small) return gateup ? launch_one<true, 2>(p, n_ctas, st) : launch_one<false, 2>(p, n_ctas, st);
-    return gateup ? launch_one<true, 3>(p, n_ctas, st) : launch_one<false, 3>(p, n_ctas, st);
+    if (small && max_rows <= 8) return gateup ? launch_one<true, 1>(p, n_ctas, G, st) : launch_one<false, 1>(p, n_ctas, G, st);
+    if (small) return gateup ? launch_one<true, 2>(p, n_ctas, G, st) : launch_one<false, 2>(p, n_ctas, G, st);
+    return gateup ? launch_one<true, 3>(p, n_ctas, G, st) : launch_one<false, 3>(p, n_ctas, G, st);
 }
 
 }  // namespace dyn
