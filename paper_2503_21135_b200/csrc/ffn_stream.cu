@@ -410,13 +410,17 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
     volatile int* poison = &S->poison;
 
     if (warp == CONSUMER_WARPS) {
-        // ---------------- producer warp: runs ahead across items ----------------
+        // ---------------- producer: ONE thread, running ahead across items.  The schedulers share the issue slots among
+        // all ready warps, so every instruction of the producer's per-stage path waits its turn behind the consumer
+        // warps of three CTAs (a per-stage timeline showed half a microsecond per stage, as long as the consumers need
+        // for it): the path is kept as short as it gets, with no warp-wide shuffles or barriers in it ----------------
+        if (lane != 0) return;
         int it = 0;
         Cursor y;
         bool ok = true;
         // byte ring: head = next write offset, tail = oldest stage not yet released, free_b = free bytes
         int head = 0, tail = 0, free_b = p.ring_bytes;
-        auto acquire = [&](int need) -> int {   // lane 0 only; returns the ring offset or -1 after an expired wait
+        auto acquire = [&](int need) -> int {   // returns the ring offset or -1 after an expired wait
             need = (need + 127) & ~127;
             int pad = 0;
             if (head + need > p.ring_bytes) { pad = p.ring_bytes - head; head = 0; }
@@ -450,17 +454,14 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
             int g = blockIdx.x;
             if (!first_draw) {
                 if (all_static) break;  // every item was dealt statically: the consumers know, nothing to signal
-                if (lane == 0) g = gridDim.x + atomicAdd(p.work_ctr, 1);
-                g = __shfl_sync(0xffffffffu, g, 0);
+                g = gridDim.x + atomicAdd(p.work_ctr, 1);
             } else if (all_static && g >= n_items) {
                 break;
             }
             first_draw = false;
             if (g >= n_items) {  // tell the consumers: an empty stage marked -1
-                int off = 0;
-                if (lane == 0) off = acquire(128);
-                off = __shfl_sync(0xffffffffu, off, 0);
-                if (off >= 0 && lane == 0) {
+                const int off = acquire(128);
+                if (off >= 0) {
                     S->first_item[it % NS] = -1;
                     mbar_arrive(&S->full[it % NS]);
                 }
@@ -477,50 +478,47 @@ __global__ void __launch_bounds__(FFN_THREADS, (MAXNT8 <= 2 && APW == 2) ? 3 : 2
             }
             const uint8_t* wbase = (GATEUP ? ex.w13 : ex.w2) + (size_t)im.rb * n_kc * blk_bytes;
             const uint8_t* xbuf = GATEUP ? p.ws.xperm : p.ws.hbuf;
+            const int stage_need = blk_bytes + ((im.nvalid + 7) & ~7) * XROW;
+            const uint32_t x_bytes = (uint32_t)(im.nvalid * XROW), stage_tx = (uint32_t)blk_bytes + x_bytes;
+            const uint8_t* wsrc = wbase + (size_t)kc0 * blk_bytes;
+            const uint8_t* xsrc = xbuf + act_off(kc0, im.row0, p.ws.Rcap);
+            const size_t x_stride = act_off(1, 0, p.ws.Rcap);   // one k chunk further in the chunk-major buffer
             for (int kc = kc0; kc < kc1 && ok; ++kc, ++it) {
                 const int s = it % NS;
-                int off = 0;
                 // the consumers read whole 8-token tiles: reserve rows up to the tile boundary (only nvalid are copied)
-                if (lane == 0) off = acquire(blk_bytes + ((im.nvalid + 7) & ~7) * XROW);
-                off = __shfl_sync(0xffffffffu, off, 0);
+                const int off = acquire(stage_need);
                 ok = off >= 0;
                 if (!ok) break;
                 uint8_t* st = stages + off;
-                if (lane == 0) {
-                    // two copies per stage: the packed block and the (chunk-major, hence contiguous) activation slice
-                    S->first_item[s] = first ? g : -2;
-                    mbar_arrive_expect_tx(&S->full[s], (uint32_t)(blk_bytes + im.nvalid * XROW));
-                    bulk_g2s(st, wbase + (size_t)kc * blk_bytes, (uint32_t)blk_bytes, &S->full[s]);
-                    bulk_g2s(st + blk_bytes, xbuf + act_off(kc, im.row0, p.ws.Rcap), (uint32_t)(im.nvalid * XROW), &S->full[s]);
-                }
+                // two copies per stage: the packed block and the (chunk-major, hence contiguous) activation slice
+                S->first_item[s] = first ? g : -2;
+                mbar_arrive_expect_tx(&S->full[s], stage_tx);
+                bulk_g2s(st, wsrc, (uint32_t)blk_bytes, &S->full[s]);
+                bulk_g2s(st + blk_bytes, xsrc, x_bytes, &S->full[s]);
+                wsrc += blk_bytes;
+                xsrc += x_stride;
                 first = false;
-                __syncwarp();
             }
             if constexpr (GATEUP) {
                 // cached-channel stages: 32 pool columns each = one 16.9 KB tile copy + one activation copy
                 const int n_ps = (ex.switchable && L->sig_cnt[im.e] > 0) ? (L->P_pad >> 5) : 0;
                 for (int ps = 0; ps < n_ps && ok; ++ps, ++it) {
                     const int s = it % NS;
-                    int off = 0;
-                    if (lane == 0) off = acquire(POOL_GROUP * POOL_TILE_PITCH + ((im.nvalid + 7) & ~7) * XPOOL_ROW);
-                    off = __shfl_sync(0xffffffffu, off, 0);
+                    const int off = acquire(POOL_GROUP * POOL_TILE_PITCH + ((im.nvalid + 7) & ~7) * XPOOL_ROW);
                     ok = off >= 0;
                     if (!ok) break;
                     uint8_t* st = stages + off;
-                    if (lane == 0) {
-                        S->first_item[s] = -2;
-                        mbar_arrive_expect_tx(&S->full[s], (uint32_t)(POOL_GROUP * POOL_TILE_PITCH + im.nvalid * XPOOL_ROW));
-                        bulk_g2s(st, reinterpret_cast<const uint8_t*>(ex.pool_hi) + pool_tile_off(im.rb, ps * POOL_GROUP, L->P_pad),
-                                 POOL_GROUP * POOL_TILE_PITCH, &S->full[s]);
-                        bulk_g2s(st + POOL_GROUP * POOL_TILE_PITCH,
-                                 reinterpret_cast<const uint8_t*>(p.ws.xsig) + xpool_off(ps, im.row0, p.ws.Rcap),
-                                 (uint32_t)(im.nvalid * XPOOL_ROW), &S->full[s]);
-                    }
-                    __syncwarp();
+                    S->first_item[s] = -2;
+                    mbar_arrive_expect_tx(&S->full[s], (uint32_t)(POOL_GROUP * POOL_TILE_PITCH + im.nvalid * XPOOL_ROW));
+                    bulk_g2s(st, reinterpret_cast<const uint8_t*>(ex.pool_hi) + pool_tile_off(im.rb, ps * POOL_GROUP, L->P_pad),
+                             POOL_GROUP * POOL_TILE_PITCH, &S->full[s]);
+                    bulk_g2s(st + POOL_GROUP * POOL_TILE_PITCH,
+                             reinterpret_cast<const uint8_t*>(p.ws.xsig) + xpool_off(ps, im.row0, p.ws.Rcap),
+                             (uint32_t)(im.nvalid * XPOOL_ROW), &S->full[s]);
                 }
             }
         }
-        if (!ok && lane == 0) {
+        if (!ok) {
             // gave up: let copies already issued land before the CTA's shared memory is released
             const unsigned long long t0 = globaltimer_ns();
             while (globaltimer_ns() - t0 < 2000000ull) {
