@@ -173,7 +173,7 @@ def time_steps(fn, steps, dist_barrier):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one gate/up launch, from the ncu captures summarised
 # under profiles/ (decode shape, layer 0); None where no capture of that launch exists.
-NCU_TRAFFIC_BYTES = {("decode", 8): 493.7e6 + 4.1e6, ("decode", 64): 496.6e6 + 8.5e6}
+NCU_TRAFFIC_BYTES = {("decode", 8): 493.8e6 + 3.8e6, ("decode", 64): 497.4e6 + 10.2e6}
 
 
 def kernel_times(layers, step_fn, steps):
