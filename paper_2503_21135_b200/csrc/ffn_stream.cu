@@ -1,12 +1,13 @@
 // Streaming grouped dequant-GEMM for small token counts per expert (decode path, and the generic
 // fallback for any size): HBM-bound, judged on packed-weight bytes per second.
 //
-// PERSISTENT grid (two CTAs per SM).  A work item = one (expert, 256-row weight block, chunk of <= 24
-// tokens, K split); items are ordered heaviest bit-width first and dealt round-robin to the CTAs, so
-// every CTA walks the same kind of mix.  Inside a CTA a producer warp streams the packed blocks (codes
-// + params, contiguous per 256 x 128 block) and the matching activation slices into a shared-memory ring
-// with bulk async copies completing on mbarriers; it runs ahead across item boundaries, so the ring
-// never drains between items.  Eight consumer warps, each owning two 16-row atoms, turn codes into fp16
+// PERSISTENT grid (two or three CTAs per SM).  A work item = one (expert, 256-row weight block, chunk of <= 24
+// tokens, K split); items are ordered costliest first (most 8-token tiles first from 33 rows per expert on, then
+// heaviest bit-width) and handed out from a device counter, a CTA's first item statically.  Inside a CTA ONE
+// producer thread streams the packed blocks (codes + params, contiguous per 256 x 128 block) and the matching
+// activation slices into a shared-memory ring with bulk async copies completing on mbarriers; it runs ahead across
+// item boundaries, so the ring never drains between items.  The group size is a template parameter (the group
+// bookkeeping of the inner loop folds away).  Eight consumer warps, each owning two 16-row atoms, turn codes into fp16
 // operands with ONE logic op per register pair: a code field masked in place at bit offset o is the
 // fp16 subnormal q * 2^(o-24), and the activation slice already carries the factor 2^(bias-o) (see
 // layout.cuh).  They issue mma.sync m16n8k16 (weights = A, tokens = B, fp32 accumulate) and apply
