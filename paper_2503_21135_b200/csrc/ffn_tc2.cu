@@ -59,7 +59,7 @@ constexpr int T2_OFF_XRING = T2_OFF_STAGE + T2_NW * T2_WHALF_MAX;
 constexpr int T2_SMEM_BYTES = T2_OFF_XRING + T2_NX * T2_XTILE;
 static_assert(T2_OFF_XRING % 1024 == 0 && T2_XTILE % 1024 == 0, "operand slots must stay 1024-byte aligned");
 static_assert(T2_OFF_PREFIX + (MAX_EXPERTS + 1) * 4 <= T2_OFF_STAGE, "item table overlaps the stage ring");
-static_assert(T2_SMEM_BYTES <= 227 * 1024, "shared memory budget");
+static_assert(T2_SMEM_BYTES <= 227 * 1024, "shared memory limit of a CTA");
 constexpr uint32_t T2_TMEM_COLS = 512;
 constexpr uint32_t T2_COL_A = 256;
 constexpr int T2_NA = 4;                               // A buffers of 64 columns: the dequant warps run ahead of the MMA
